@@ -1,0 +1,204 @@
+/*
+ * cobs.h -- C ABI of the COBS (Cumulant Order Block Sparse attention) decode path for NVIDIA B200.
+ *
+ * One decode step of one attention layer, for a batch of sequences whose keys and
+ * values live in a paged bf16 KV cache:
+ *
+ *   (a) cobs_build_summaries   per KV block: mean key, and the top-r scaled eigenvectors of the
+ *                              within-block key covariance (full key space or a query subspace),
+ *                              stored as fp32, bf16 or FP4 E2M1 with one scale per eigenvector
+ *   (b,c) cobs_score_select    second-order estimate of every block's log attention mass for each
+ *                              query head, the GQA group score, and the top-k blocks per KV head
+ *   (d) cobs_sparse_decode     softmax attention over the selected blocks plus a local window
+ *   fused: cobs_decode_step    (b) (c) (d) in one call
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a parameter is named *_host.
+ *     The library allocates no device memory and frees none; scratch comes from the caller as
+ *     `workspace` (size from cobs_workspace_bytes, 256-byte aligned).  The workspace must not be
+ *     shared by calls that may overlap on the GPU.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     the call returns without synchronising, except the *_host entry point and cobs_read_status.
+ *   - Arguments are validated on the host before anything is launched; a call that returns a
+ *     nonzero status has launched nothing.
+ *   - Device-side problems (an index outside its array, a bounded wait that ran out) do not fault:
+ *     the kernel skips the access, records a code in the status word at the start of the workspace,
+ *     and cobs_read_status returns it.
+ *   - Shapes: B sequences, Hq query heads, Hkv KV heads, G = Hq/Hkv, head dimension D, block of L
+ *     tokens, page of P tokens (P divides L), r stored eigenvectors, Ds = sub_dim or D.
+ *   - The attention scale 1/sqrt(D) is folded into the query inside the library (the paper's
+ *     Notation paragraph absorbs it into q); callers pass the raw query.
+ *
+ * Block / window rule (one per sequence of length T):
+ *   summarised blocks   b < floor(T / L)          (only full blocks have summaries)
+ *   window              tokens [ws, T), ws = floor(max(0, T - window) / L) * L
+ *   candidates          blocks b < ws / L        (wholly before the window)
+ *   selected            min(topk, ws / L) candidates with the largest group score; larger score
+ *                       first, lower block index on equal scores; reported in ascending index
+ *                       order, padded with -1.
+ */
+#ifndef COBS_H_
+#define COBS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  COBS_OK = 0,
+  COBS_ERR_INVALID_ARG = 1,         /* NULL pointer, misaligned pointer, inconsistent or out-of-range field */
+  COBS_ERR_UNSUPPORTED = 2,         /* a shape this build has no kernel for */
+  COBS_ERR_WORKSPACE_TOO_SMALL = 3,
+  COBS_ERR_CUDA = 4,                /* a CUDA runtime call failed (launch configuration, copy) */
+  COBS_ERR_TIMEOUT = 5,             /* device status: a bounded device-side wait ran out */
+  COBS_ERR_BOUNDS = 6               /* device status: a page id or block index was out of range and skipped */
+} cobs_status;
+
+typedef enum { COBS_SUMM_FP32 = 0, COBS_SUMM_BF16 = 1, COBS_SUMM_FP4_E2M1 = 2 } cobs_summary_dtype;
+typedef enum { COBS_SCALE_FP32 = 0, COBS_SCALE_FP16 = 1 } cobs_scale_dtype;
+
+#define COBS_MAX_TOPK 128
+#define COBS_MAX_RANK 16
+
+/* Problem statement: shapes and method parameters (paper: Background, Notation; Method). */
+typedef struct {
+  int32_t batch;              /* B >= 1 */
+  int32_t n_q_heads;          /* Hq, a multiple of n_kv_heads; G = Hq / Hkv in {1, 2, 4, 8} */
+  int32_t n_kv_heads;         /* Hkv >= 1 */
+  int32_t head_dim;           /* D in {64, 128} */
+  int32_t block_size;         /* L in {16, 32, 64, 128} */
+  int32_t page_size;          /* P: tokens per KV page; >= 16, divides L or equals L */
+  int32_t rank;               /* r in 0..COBS_MAX_RANK; 0 = first-order (mean-pool) score */
+  int32_t sub_dim;            /* 0 = full-space descriptor (Ds = D); else Ds in [8, D], u_q required */
+  int32_t topk;               /* k in 1..COBS_MAX_TOPK */
+  int32_t window;             /* local window in tokens, >= 1 */
+  int32_t summary_dtype;      /* cobs_summary_dtype */
+  int32_t scale_dtype;        /* cobs_scale_dtype; read only when summary_dtype == COBS_SUMM_FP4_E2M1 */
+  int32_t max_blocks;         /* NB: block capacity per sequence = stride of the summary arrays */
+  int32_t max_pages_per_seq;  /* row stride of page_table */
+} cobs_config;
+
+/* Paged bf16 KV cache. */
+typedef struct {
+  const void *k_pages;        /* [n_pages][Hkv][P][D] bf16 */
+  const void *v_pages;        /* [n_pages][Hkv][P][D] bf16 */
+  const int32_t *page_table;  /* [B][max_pages_per_seq]: page id of the i-th page of a sequence */
+  const int32_t *seq_lens;    /* [B]: tokens in the cache, the current one included; 1 <= T <= NB*L + L - 1 */
+  int64_t n_pages;            /* page ids are checked against this */
+} cobs_kv;
+
+/*
+ * Per-block summaries (paper: Method, second-order truncation, covariance compression, subspace
+ * method, quantization).  Layout per (sequence, KV head, block):
+ *   mean   [B][Hkv][NB][D]                fp32 (COBS_SUMM_FP32) or bf16 (BF16 and FP4 modes)
+ *   xi     [B][Hkv][NB][r][Ds]            fp32 | bf16, or for FP4 [B][Hkv][NB][r * Ds_pad / 2] bytes:
+ *                                         E2M1 codes (bit 3 sign, bits 2..0 magnitude index into
+ *                                         {0, .5, 1, 1.5, 2, 3, 4, 6}), element 2j of a row in the low
+ *                                         nibble of byte j, element 2j+1 in the high nibble; rows are
+ *                                         Ds_pad = cobs_padded_sub_dim() elements long, padding codes 0
+ *   scale  [B][Hkv][NB][r]                fp32 | fp16, FP4 mode only: xi_hat = magnitude * scale
+ *   u_q    [Hkv][D][Ds] fp32              orthonormal columns spanning the query subspace; NULL when
+ *                                         sub_dim == 0
+ */
+typedef struct {
+  void *mean;
+  void *xi;
+  void *scale;
+  const float *u_q;
+} cobs_summaries;
+
+const char *cobs_status_string(int32_t status);
+
+/* Row length in elements of a packed FP4 factor row: Ds rounded up so that every block's factor record
+ * (r rows) is a whole number of 16-byte units and every row a whole number of 4-byte words. */
+int32_t cobs_padded_sub_dim(const cobs_config *cfg);
+
+/* Bytes of each summary array for cfg (scale_bytes = 0 unless FP4).  Host-only arithmetic. */
+int32_t cobs_summary_bytes(const cobs_config *cfg, size_t *mean_bytes, size_t *xi_bytes, size_t *scale_bytes);
+
+/* Bytes of workspace that any entry point needs for cfg. */
+int32_t cobs_workspace_bytes(const cobs_config *cfg, size_t *bytes);
+
+/* Zero the status word of a workspace (enqueued on stream).  Call once after allocating it. */
+int32_t cobs_reset_status(void *workspace, size_t workspace_bytes, void *stream);
+
+/* Synchronise `stream`, copy the status word to *code_host (COBS_OK, COBS_ERR_TIMEOUT or COBS_ERR_BOUNDS). */
+int32_t cobs_read_status(void *workspace, size_t workspace_bytes, void *stream, int32_t *code_host);
+
+/*
+ * (a) Build the summaries of blocks [block_begin, block_end) of every sequence and KV head; per
+ * sequence the range is clipped to the full blocks, floor(T / L).
+ *   mean   = (1/L) sum_t k_t                         (Eq. cgf-cumulants)
+ *   K~     = rows k_t - mean (un-rounded mean), times U_Q when sub_dim > 0
+ *   C      = K~ K~^T / L, eigenpairs (lambda_i, w_i), lambda descending
+ *   xi_i   = K~^T w_i / sqrt(L), i < r                (Method, Cost: Gram trick; Eq. lowrank)
+ *            sign: the entry of largest magnitude is positive; a direction whose eigenvalue is below
+ *            1e-12 of the block's mean squared key norm is stored as zeros
+ *   store  : fp32 / bf16 (round to nearest even) / FP4 as cobs_quantise_xi does
+ * Arithmetic is fp32.  Deterministic: the same input gives the same bits.
+ */
+int32_t cobs_build_summaries(const cobs_config *cfg, const cobs_kv *kv, int32_t block_begin, int32_t block_end,
+                             const cobs_summaries *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The FP4 quantiser of step (a) on its own (Method, Quantization: E2M1, one scale per eigenvector).
+ * xi_fp32 [n_vectors][Ds] -> codes [n_vectors][Ds_pad / 2] bytes, scale [n_vectors] (cfg->scale_dtype).
+ *   a = max |xi_j|; scale = a / 6 (fp32 division; rounded to fp16 when the scale is fp16);
+ *   t_j = xi_j / scale (fp32 division); code = sign bit of xi_j, nearest E2M1 magnitude to |t_j|,
+ *   ties to the even mantissa bit, saturating at 6; scale 0 -> all codes 0.
+ * Reads cfg->head_dim, sub_dim, rank, scale_dtype only.  n_vectors must be a multiple of cfg->rank.
+ */
+int32_t cobs_quantise_xi(const cobs_config *cfg, const float *xi_fp32, int64_t n_vectors, void *codes, void *scale,
+                         void *stream);
+
+/*
+ * (b) + (c) Score every summarised block and select (Eq. trunc, Eq. gram, Eq. gqa-secondorder).
+ *   q' = q / sqrt(D);  q~ = U_Q^T q' (or q')
+ *   e[g][b]  = ln L + q'_g . mean_b + 1/2 sum_i (xi_{b,i} . q~_g)^2
+ *   score[b] = sum_g exp(e[g][b] - logsumexp_b' e[g][b'])       over all summarised blocks b'
+ * q        [B][Hq][D] bf16
+ * sel_idx  [B][Hkv][topk] int32 out, ascending, padded with -1
+ * sel_cnt  [B][Hkv] int32 out
+ * scores_or_null [B][Hkv][NB] fp32 out (entries b >= floor(T/L) are left untouched)
+ */
+int32_t cobs_score_select(const cobs_config *cfg, const void *q, const cobs_summaries *summ, const int32_t *seq_lens,
+                          int32_t *sel_idx, int32_t *sel_cnt, float *scores_or_null, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
+/*
+ * (d) Attention over the selected blocks and the window, one softmax over their union
+ * (Eq. oracle-true restricted to the kept blocks and the window).
+ * out [B][Hq][D] fp32; lse_or_null [B][Hq] fp32 = log of the softmax denominator (natural log).
+ * sel_idx entries must be distinct candidate blocks in [0, ws/L); others are skipped and reported
+ * as COBS_ERR_BOUNDS in the status word.
+ */
+int32_t cobs_sparse_decode(const cobs_config *cfg, const void *q, const cobs_kv *kv, const int32_t *sel_idx,
+                           const int32_t *sel_cnt, float *out, float *lse_or_null, void *workspace,
+                           size_t workspace_bytes, void *stream);
+
+/*
+ * Fused step: cobs_score_select followed by cobs_sparse_decode on its selection.
+ * sel_idx_or_null / sel_cnt_or_null receive the selection when given.
+ */
+int32_t cobs_decode_step(const cobs_config *cfg, const void *q, const cobs_kv *kv, const cobs_summaries *summ,
+                         float *out, float *lse_or_null, int32_t *sel_idx_or_null, int32_t *sel_cnt_or_null,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The fused step for a caller whose per-step tensors live in HOST memory: copies q_host to the device,
+ * runs cobs_decode_step, copies the output back and synchronises `stream`.  The KV cache, page table and
+ * summaries stay on the device (they are the state a decode loop keeps there).  q_host [B][Hq][D] bf16 and
+ * out_host [B][Hq][D] fp32 should be pinned for the copies to be asynchronous; sel_idx_host_or_null
+ * [B][Hkv][topk] and sel_cnt_host_or_null [B][Hkv] receive the selection when given.
+ */
+int32_t cobs_decode_step_host(const cobs_config *cfg, const void *q_host, const cobs_kv *kv,
+                              const cobs_summaries *summ, float *out_host, int32_t *sel_idx_host_or_null,
+                              int32_t *sel_cnt_host_or_null, void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COBS_H_ */

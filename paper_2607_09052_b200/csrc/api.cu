@@ -1,0 +1,306 @@
+// Host side of the C ABI: argument validation, workspace carving, kernel launches.
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace cobs {
+cudaError_t launch_score(const Params &p, cudaStream_t stream);
+cudaError_t launch_select(const Params &p, cudaStream_t stream);
+cudaError_t launch_attend(const Params &p, cudaStream_t stream);
+cudaError_t launch_build(const Params &p, int block_begin, int block_end, cudaStream_t stream);
+cudaError_t launch_quantise(const float *xi, long long n_vectors, int Ds, int Ds_pad, int scale_dtype, void *codes,
+                            void *scale, cudaStream_t stream);
+size_t build_smem_bytes(const Params &p);
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int padded_sub_dim(int Ds, int r) {
+  int pad = (Ds + 7) / 8 * 8;
+  if (r > 0)
+    while (((size_t)r * pad / 2) % 16 != 0) pad += 8;
+  return pad;
+}
+
+static bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+static int32_t validate_config(const cobs_config *c) {
+  if (!c) return COBS_ERR_INVALID_ARG;
+  if (c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return COBS_ERR_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads != 0) return COBS_ERR_INVALID_ARG;
+  const int G = c->n_q_heads / c->n_kv_heads;
+  if (!(G == 1 || G == 2 || G == 4 || G == 8)) return COBS_ERR_UNSUPPORTED;
+  if (!(c->head_dim == 64 || c->head_dim == 128)) return COBS_ERR_UNSUPPORTED;
+  if (!is_pow2(c->block_size) || c->block_size < 16 || c->block_size > 128) return COBS_ERR_UNSUPPORTED;
+  if (!is_pow2(c->page_size) || c->page_size < 16 || c->page_size > c->block_size) return COBS_ERR_INVALID_ARG;
+  if (c->rank < 0 || c->rank > COBS_MAX_RANK) return COBS_ERR_INVALID_ARG;
+  if (c->sub_dim != 0 && (c->sub_dim < 8 || c->sub_dim > c->head_dim)) return COBS_ERR_INVALID_ARG;
+  if (c->topk < 1 || c->topk > COBS_MAX_TOPK) return COBS_ERR_INVALID_ARG;
+  if (c->window < 1) return COBS_ERR_INVALID_ARG;
+  if (c->summary_dtype < COBS_SUMM_FP32 || c->summary_dtype > COBS_SUMM_FP4_E2M1) return COBS_ERR_INVALID_ARG;
+  if (c->summary_dtype == COBS_SUMM_FP4_E2M1 && c->scale_dtype != COBS_SCALE_FP32 && c->scale_dtype != COBS_SCALE_FP16)
+    return COBS_ERR_INVALID_ARG;
+  if (c->max_blocks < 1 || c->max_blocks > (1 << 20)) return COBS_ERR_INVALID_ARG;
+  if (c->max_pages_per_seq < 1) return COBS_ERR_INVALID_ARG;
+  // the page table must cover every token a sequence may hold: NB * L + L - 1 at most
+  if ((long long)c->max_pages_per_seq * c->page_size < (long long)c->max_blocks * c->block_size) return COBS_ERR_INVALID_ARG;
+  return COBS_OK;
+}
+
+static int choose_splits(const cobs_config *c) {
+  const int units = c->batch * c->n_kv_heads;
+  const int items = c->topk + (c->window + c->block_size - 1) / c->block_size + 1;
+  int s = (2 * 148 + units - 1) / units;
+  if (s > items) s = items;
+  if (s > kMaxSplits) s = kMaxSplits;
+  if (s < 1) s = 1;
+  return s;
+}
+
+struct WorkspaceLayout {
+  size_t status, e, partial, sel_idx, sel_cnt, q_stage, out_stage, total;
+};
+
+static WorkspaceLayout layout_workspace(const cobs_config *c) {
+  WorkspaceLayout w;
+  const size_t B = c->batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, G = Hq / Hkv, D = c->head_dim;
+  size_t off = 0;
+  w.status = off; off += kStatusBytes;
+  w.e = off; off = align_up(off + B * Hq * (size_t)c->max_blocks * sizeof(float), 256);
+  w.partial = off; off = align_up(off + B * Hkv * (size_t)choose_splits(c) * G * (D + 2) * sizeof(float), 256);
+  w.sel_idx = off; off = align_up(off + B * Hkv * (size_t)c->topk * sizeof(int32_t), 256);
+  w.sel_cnt = off; off = align_up(off + B * Hkv * sizeof(int32_t), 256);
+  w.q_stage = off; off = align_up(off + B * Hq * D * 2, 256);
+  w.out_stage = off; off = align_up(off + B * Hq * D * sizeof(float), 256);
+  w.total = off;
+  return w;
+}
+
+static void fill_params(Params &p, const cobs_config *c, void *workspace) {
+  memset(&p, 0, sizeof(p));
+  p.B = c->batch; p.Hq = c->n_q_heads; p.Hkv = c->n_kv_heads; p.G = p.Hq / p.Hkv; p.D = c->head_dim;
+  p.L = c->block_size; p.P = c->page_size; p.r = c->rank;
+  p.Ds = c->sub_dim ? c->sub_dim : c->head_dim;
+  p.Ds_pad = (c->summary_dtype == COBS_SUMM_FP4_E2M1) ? padded_sub_dim(p.Ds, p.r) : p.Ds;
+  p.topk = c->topk; p.window = c->window; p.NB = c->max_blocks; p.mpp = c->max_pages_per_seq;
+  p.summ_dtype = c->summary_dtype; p.scale_dtype = c->scale_dtype;
+  p.n_splits = choose_splits(c);
+  if (workspace) {
+    WorkspaceLayout w = layout_workspace(c);
+    char *base = static_cast<char *>(workspace);
+    p.status = reinterpret_cast<int32_t *>(base + w.status);
+    p.e = reinterpret_cast<float *>(base + w.e);
+    p.partial = reinterpret_cast<float *>(base + w.partial);
+    p.sel_idx = reinterpret_cast<int32_t *>(base + w.sel_idx);
+    p.sel_cnt = reinterpret_cast<int32_t *>(base + w.sel_cnt);
+  }
+}
+
+static int32_t check_workspace(const cobs_config *c, void *workspace, size_t bytes) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return COBS_ERR_INVALID_ARG;
+  if (bytes < layout_workspace(c).total) return COBS_ERR_WORKSPACE_TOO_SMALL;
+  return COBS_OK;
+}
+
+static int32_t set_summaries(Params &p, const cobs_config *c, const cobs_summaries *s) {
+  if (!s || !s->mean || !aligned16(s->mean)) return COBS_ERR_INVALID_ARG;
+  if (c->rank > 0 && (!s->xi || !aligned16(s->xi))) return COBS_ERR_INVALID_ARG;
+  if (c->rank > 0 && c->summary_dtype == COBS_SUMM_FP4_E2M1 && (!s->scale || !aligned16(s->scale)))
+    return COBS_ERR_INVALID_ARG;
+  if (c->sub_dim != 0 && (!s->u_q || !aligned16(s->u_q))) return COBS_ERR_INVALID_ARG;
+  p.mean = s->mean; p.xi = s->xi; p.scale = s->scale;
+  p.u_q = c->sub_dim ? s->u_q : nullptr;
+  return COBS_OK;
+}
+
+static int32_t set_kv(Params &p, const cobs_kv *kv) {
+  if (!kv || !kv->k_pages || !kv->v_pages || !kv->page_table || !kv->seq_lens || kv->n_pages < 1)
+    return COBS_ERR_INVALID_ARG;
+  if (!aligned16(kv->k_pages) || !aligned16(kv->v_pages)) return COBS_ERR_INVALID_ARG;
+  p.k_pages = static_cast<const __nv_bfloat16 *>(kv->k_pages);
+  p.v_pages = static_cast<const __nv_bfloat16 *>(kv->v_pages);
+  p.page_table = kv->page_table; p.seq_lens = kv->seq_lens; p.n_pages = kv->n_pages;
+  return COBS_OK;
+}
+
+static int32_t cuda_status(cudaError_t e) { return e == cudaSuccess ? COBS_OK : COBS_ERR_CUDA; }
+
+}  // namespace cobs
+
+using namespace cobs;
+
+extern "C" {
+
+const char *cobs_status_string(int32_t s) {
+  switch (s) {
+    case COBS_OK: return "ok";
+    case COBS_ERR_INVALID_ARG: return "invalid argument";
+    case COBS_ERR_UNSUPPORTED: return "unsupported shape";
+    case COBS_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case COBS_ERR_CUDA: return "CUDA runtime error";
+    case COBS_ERR_TIMEOUT: return "device-side wait ran out";
+    case COBS_ERR_BOUNDS: return "index out of range on the device (access skipped)";
+    default: return "unknown status";
+  }
+}
+
+int32_t cobs_padded_sub_dim(const cobs_config *cfg) {
+  if (validate_config(cfg) != COBS_OK) return -1;
+  return padded_sub_dim(cfg->sub_dim ? cfg->sub_dim : cfg->head_dim, cfg->rank);
+}
+
+int32_t cobs_summary_bytes(const cobs_config *cfg, size_t *mean_bytes, size_t *xi_bytes, size_t *scale_bytes) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if (!mean_bytes || !xi_bytes || !scale_bytes) return COBS_ERR_INVALID_ARG;
+  const size_t n = (size_t)cfg->batch * cfg->n_kv_heads * cfg->max_blocks;
+  const int Ds = cfg->sub_dim ? cfg->sub_dim : cfg->head_dim;
+  switch (cfg->summary_dtype) {
+    case COBS_SUMM_FP32:
+      *mean_bytes = n * cfg->head_dim * 4; *xi_bytes = n * cfg->rank * Ds * 4; *scale_bytes = 0; break;
+    case COBS_SUMM_BF16:
+      *mean_bytes = n * cfg->head_dim * 2; *xi_bytes = n * cfg->rank * Ds * 2; *scale_bytes = 0; break;
+    default:
+      *mean_bytes = n * cfg->head_dim * 2;
+      *xi_bytes = n * cfg->rank * (padded_sub_dim(Ds, cfg->rank) / 2);
+      *scale_bytes = n * cfg->rank * (cfg->scale_dtype == COBS_SCALE_FP16 ? 2 : 4);
+      break;
+  }
+  return COBS_OK;
+}
+
+int32_t cobs_workspace_bytes(const cobs_config *cfg, size_t *bytes) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if (!bytes) return COBS_ERR_INVALID_ARG;
+  *bytes = layout_workspace(cfg).total;
+  return COBS_OK;
+}
+
+int32_t cobs_reset_status(void *workspace, size_t workspace_bytes, void *stream) {
+  if (!workspace || workspace_bytes < (size_t)kStatusBytes) return COBS_ERR_INVALID_ARG;
+  return cuda_status(cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t cobs_read_status(void *workspace, size_t workspace_bytes, void *stream, int32_t *code_host) {
+  if (!workspace || workspace_bytes < (size_t)kStatusBytes || !code_host) return COBS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(code_host, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return COBS_ERR_CUDA;
+  return cuda_status(cudaStreamSynchronize(s));
+}
+
+int32_t cobs_build_summaries(const cobs_config *cfg, const cobs_kv *kv, int32_t block_begin, int32_t block_end,
+                             const cobs_summaries *out, void *workspace, size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (block_begin < 0 || block_end < block_begin || block_end > cfg->max_blocks) return COBS_ERR_INVALID_ARG;
+  Params p;
+  fill_params(p, cfg, workspace);
+  if ((st = set_kv(p, kv)) != COBS_OK) return st;
+  if ((st = set_summaries(p, cfg, out)) != COBS_OK) return st;
+  if (build_smem_bytes(p) > 227 * 1024) return COBS_ERR_UNSUPPORTED;
+  return cuda_status(launch_build(p, block_begin, block_end, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t cobs_quantise_xi(const cobs_config *cfg, const float *xi_fp32, int64_t n_vectors, void *codes, void *scale,
+                         void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if (!xi_fp32 || !codes || !scale || n_vectors < 0 || cfg->rank < 1 || n_vectors % cfg->rank != 0)
+    return COBS_ERR_INVALID_ARG;
+  if (!aligned16(codes) || !aligned16(scale) || !aligned16(xi_fp32)) return COBS_ERR_INVALID_ARG;
+  const int Ds = cfg->sub_dim ? cfg->sub_dim : cfg->head_dim;
+  return cuda_status(launch_quantise(xi_fp32, n_vectors, Ds, padded_sub_dim(Ds, cfg->rank), cfg->scale_dtype, codes,
+                                     scale, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t cobs_score_select(const cobs_config *cfg, const void *q, const cobs_summaries *summ, const int32_t *seq_lens,
+                          int32_t *sel_idx, int32_t *sel_cnt, float *scores_or_null, void *workspace,
+                          size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (!q || !aligned16(q) || !seq_lens || !sel_idx || !sel_cnt) return COBS_ERR_INVALID_ARG;
+  Params p;
+  fill_params(p, cfg, workspace);
+  if ((st = set_summaries(p, cfg, summ)) != COBS_OK) return st;
+  p.q = static_cast<const __nv_bfloat16 *>(q);
+  p.seq_lens = seq_lens;
+  p.sel_idx = sel_idx; p.sel_cnt = sel_cnt; p.scores = scores_or_null;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_score(p, s);
+  if (e != cudaSuccess) return COBS_ERR_CUDA;
+  return cuda_status(launch_select(p, s));
+}
+
+int32_t cobs_sparse_decode(const cobs_config *cfg, const void *q, const cobs_kv *kv, const int32_t *sel_idx,
+                           const int32_t *sel_cnt, float *out, float *lse_or_null, void *workspace,
+                           size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (!q || !aligned16(q) || !sel_idx || !sel_cnt || !out || !aligned16(out)) return COBS_ERR_INVALID_ARG;
+  Params p;
+  fill_params(p, cfg, workspace);
+  if ((st = set_kv(p, kv)) != COBS_OK) return st;
+  p.q = static_cast<const __nv_bfloat16 *>(q);
+  p.sel_idx = const_cast<int32_t *>(sel_idx); p.sel_cnt = const_cast<int32_t *>(sel_cnt);
+  p.out = out; p.lse = lse_or_null;
+  return cuda_status(launch_attend(p, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t cobs_decode_step(const cobs_config *cfg, const void *q, const cobs_kv *kv, const cobs_summaries *summ,
+                         float *out, float *lse_or_null, int32_t *sel_idx_or_null, int32_t *sel_cnt_or_null,
+                         void *workspace, size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (!q || !aligned16(q) || !out || !aligned16(out)) return COBS_ERR_INVALID_ARG;
+  if ((sel_idx_or_null == nullptr) != (sel_cnt_or_null == nullptr)) return COBS_ERR_INVALID_ARG;
+  Params p;
+  fill_params(p, cfg, workspace);
+  if ((st = set_kv(p, kv)) != COBS_OK) return st;
+  if ((st = set_summaries(p, cfg, summ)) != COBS_OK) return st;
+  p.q = static_cast<const __nv_bfloat16 *>(q);
+  if (sel_idx_or_null) { p.sel_idx = sel_idx_or_null; p.sel_cnt = sel_cnt_or_null; }
+  p.out = out; p.lse = lse_or_null;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_score(p, s);
+  if (e != cudaSuccess) return COBS_ERR_CUDA;
+  if ((e = launch_select(p, s)) != cudaSuccess) return COBS_ERR_CUDA;
+  return cuda_status(launch_attend(p, s));
+}
+
+int32_t cobs_decode_step_host(const cobs_config *cfg, const void *q_host, const cobs_kv *kv,
+                              const cobs_summaries *summ, float *out_host, int32_t *sel_idx_host_or_null,
+                              int32_t *sel_cnt_host_or_null, void *workspace, size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (!q_host || !out_host) return COBS_ERR_INVALID_ARG;
+  if ((sel_idx_host_or_null == nullptr) != (sel_cnt_host_or_null == nullptr)) return COBS_ERR_INVALID_ARG;
+  WorkspaceLayout w = layout_workspace(cfg);
+  char *base = static_cast<char *>(workspace);
+  void *q_dev = base + w.q_stage;
+  float *out_dev = reinterpret_cast<float *>(base + w.out_stage);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t n = (size_t)cfg->batch * cfg->n_q_heads * cfg->head_dim;
+  if (cudaMemcpyAsync(q_dev, q_host, n * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return COBS_ERR_CUDA;
+  st = cobs_decode_step(cfg, q_dev, kv, summ, out_dev, nullptr, nullptr, nullptr, workspace, workspace_bytes, stream);
+  if (st != COBS_OK) return st;
+  if (cudaMemcpyAsync(out_host, out_dev, n * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return COBS_ERR_CUDA;
+  if (sel_idx_host_or_null) {
+    const size_t units = (size_t)cfg->batch * cfg->n_kv_heads;
+    if (cudaMemcpyAsync(sel_idx_host_or_null, base + w.sel_idx, units * cfg->topk * sizeof(int32_t),
+                        cudaMemcpyDeviceToHost, s) != cudaSuccess) return COBS_ERR_CUDA;
+    if (cudaMemcpyAsync(sel_cnt_host_or_null, base + w.sel_cnt, units * sizeof(int32_t), cudaMemcpyDeviceToHost,
+                        s) != cudaSuccess) return COBS_ERR_CUDA;
+  }
+  return cuda_status(cudaStreamSynchronize(s));
+}
+
+}  // extern "C"

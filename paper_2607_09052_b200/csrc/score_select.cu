@@ -1,0 +1,272 @@
+// Steps (b) and (c): second-order block scores from the stored summaries, GQA group score, top-k.
+//
+//   e[g][b]  = ln L + q'_g . mean_b + 1/2 sum_i (xi_{b,i} . q~_g)^2      (Eq. trunc with Eq. gram)
+//   score[b] = sum_g exp(e[g][b] - logsumexp_b' e[g][b'])                (Eq. gqa-secondorder)
+//   selection: k largest scores among the candidate blocks, lower index on ties, ascending output.
+#include "common.cuh"
+
+namespace cobs {
+
+// ------------------------------------------------------------------------------------------------
+// Query preparation shared by the scoring kernels: q' = q / sqrt(D) and q~ = U_Q^T q' (or q').
+// qs: [G][D], qt: [G][Ds_pad] (zero padded), both in shared memory.
+// ------------------------------------------------------------------------------------------------
+template <int G>
+__device__ void prepare_query(const Params &p, int b_idx, int h, float *qs, float *qt) {
+  const float inv_sqrt_d = 1.0f / sqrtf((float)p.D);
+  for (int i = threadIdx.x; i < G * p.D; i += blockDim.x) {
+    int g = i / p.D, d = i - g * p.D;
+    qs[i] = __bfloat162float(p.q[((size_t)b_idx * p.Hq + h * G + g) * p.D + d]) * inv_sqrt_d;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < G * p.Ds_pad; i += blockDim.x) {
+    int g = i / p.Ds_pad, s = i - g * p.Ds_pad;
+    float v = 0.f;
+    if (s < p.Ds) {
+      if (p.u_q) {
+        const float *u = p.u_q + (size_t)h * p.D * p.Ds + s;
+        for (int d = 0; d < p.D; ++d) v = fmaf(u[(size_t)d * p.Ds], qs[g * p.D + d], v);
+      } else {
+        v = qs[g * p.D + s];
+      }
+    }
+    qt[i] = v;
+  }
+  __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Generic scoring kernel (any summary dtype, any Ds): one warp per block record, lanes stride the
+// row, fp32 FMA, warp-shuffle reduction per (row, head).
+// grid = (ceil(NB / blocks_per_cta), B * Hkv), block = 256 threads.
+// ------------------------------------------------------------------------------------------------
+template <int G, int DT>
+__global__ void __launch_bounds__(256) score_generic_kernel(Params p, int blocks_per_cta) {
+  extern __shared__ float smem[];
+  float *qs = smem;                 // [G][D]
+  float *qt = smem + G * p.D;       // [G][Ds_pad]
+  const int u = blockIdx.y, b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
+  int T = p.seq_lens[b_idx];
+  int n_sum = min(T / p.L, p.NB);
+  const int first = blockIdx.x * blocks_per_cta;
+  if (first >= n_sum) return;
+  prepare_query<G>(p, b_idx, h, qs, qt);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  const int last = min(first + blocks_per_cta, n_sum);
+  const float ln_l = logf((float)p.L);
+  for (int b = first + warp; b < last; b += n_warps) {
+    const size_t rec = (size_t)u * p.NB + b;
+    float acc[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) acc[g] = 0.f;
+    // first-order term: q' . mean
+    for (int j = lane; j < p.D; j += 32) {
+      float m = (DT == COBS_SUMM_FP32) ? ((const float *)p.mean)[rec * p.D + j]
+                                       : __bfloat162float(((const __nv_bfloat16 *)p.mean)[rec * p.D + j]);
+#pragma unroll
+      for (int g = 0; g < G; ++g) acc[g] = fmaf(m, qs[g * p.D + j], acc[g]);
+    }
+    float first_order[G], second[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) { first_order[g] = warp_sum(acc[g]); second[g] = 0.f; }
+    // curvature term from the r stored factors
+    for (int i = 0; i < p.r; ++i) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) acc[g] = 0.f;
+      float sc = 1.0f;
+      if (DT == COBS_SUMM_FP4_E2M1) {
+        sc = (p.scale_dtype == COBS_SCALE_FP16) ? __half2float(((const __half *)p.scale)[rec * p.r + i])
+                                                : ((const float *)p.scale)[rec * p.r + i];
+      }
+      for (int j = lane; j < p.Ds; j += 32) {
+        float x;
+        if (DT == COBS_SUMM_FP32) {
+          x = ((const float *)p.xi)[(rec * p.r + i) * p.Ds + j];
+        } else if (DT == COBS_SUMM_BF16) {
+          x = __bfloat162float(((const __nv_bfloat16 *)p.xi)[(rec * p.r + i) * p.Ds + j]);
+        } else {
+          uint32_t byte = ((const uint8_t *)p.xi)[(rec * p.r + i) * (size_t)(p.Ds_pad / 2) + (j >> 1)];
+          x = e2m1_value((j & 1) ? (byte >> 4) : (byte & 15u));
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) acc[g] = fmaf(x, qt[g * p.Ds_pad + j], acc[g]);
+      }
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float d = warp_sum(acc[g]) * sc;
+        second[g] = fmaf(d, d, second[g]);
+      }
+    }
+    if (lane < G) {
+      float v = 0.f;
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+        if (lane == g) v = ln_l + first_order[g] + 0.5f * second[g];
+      p.e[((size_t)u * G + lane) * p.NB + b] = v;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Group score + top-k, one CTA per (sequence, KV head).
+// ------------------------------------------------------------------------------------------------
+constexpr int kSelThreads = 256;
+
+__device__ float block_reduce(float v, bool is_max, float *scratch) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  v = is_max ? warp_max(v) : warp_sum(v);
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  float r = scratch[0];
+  for (int w = 1; w < (int)(blockDim.x >> 5); ++w) r = is_max ? fmaxf(r, scratch[w]) : r + scratch[w];
+  return r;
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_kernel(Params p) {
+  extern __shared__ float score[];                 // [NB]
+  __shared__ float scratch[kSelThreads / 32];
+  __shared__ float lse[8];
+  __shared__ int hist[256];
+  __shared__ int counts[kSelThreads];
+  __shared__ int eq_base[kSelThreads];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_need;
+
+  const int u = blockIdx.x, b_idx = u / p.Hkv, tid = threadIdx.x;
+  const int T = p.seq_lens[b_idx];
+  const int n_sum = min(T / p.L, p.NB);
+  const int n_cand = min(window_start(T, p.window, p.L) / p.L, n_sum);
+  const int G = p.G;
+
+  // log-sum-exp of each head's estimates over every summarised block
+  for (int g = 0; g < G; ++g) {
+    const float *e = p.e + ((size_t)u * G + g) * p.NB;
+    float mx = -INFINITY;
+    for (int b = tid; b < n_sum; b += kSelThreads) mx = fmaxf(mx, e[b]);
+    mx = block_reduce(mx, true, scratch);
+    float sm = 0.f;
+    for (int b = tid; b < n_sum; b += kSelThreads) sm += expf(e[b] - mx);
+    sm = block_reduce(sm, false, scratch);
+    if (tid == 0) lse[g] = mx + logf(sm);
+  }
+  __syncthreads();
+  for (int b = tid; b < n_sum; b += kSelThreads) {
+    float s = 0.f;
+    for (int g = 0; g < G; ++g) s += expf(p.e[((size_t)u * G + g) * p.NB + b] - lse[g]);
+    score[b] = s;
+    if (p.scores) p.scores[(size_t)u * p.NB + b] = s;
+  }
+  __syncthreads();
+
+  int32_t *out = p.sel_idx + (size_t)u * p.topk;
+  const int k = min(p.topk, n_cand);
+  if (tid == 0) p.sel_cnt[u] = k;
+  for (int i = k + tid; i < p.topk; i += kSelThreads) out[i] = -1;
+  if (k == 0) return;
+  if (k == n_cand) {
+    for (int i = tid; i < k; i += kSelThreads) out[i] = i;
+    return;
+  }
+
+  // radix select of the k-th largest key (scores are >= 0, so their bit patterns order like integers)
+  if (tid == 0) { s_prefix = 0u; s_need = k; }
+  uint32_t mask = 0u;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    for (int b = tid; b < n_cand; b += kSelThreads) {
+      uint32_t key = __float_as_uint(score[b]);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int need = s_need, cum = 0, bin = 255;
+      for (; bin > 0; --bin) {
+        if (cum + hist[bin] >= need) break;
+        cum += hist[bin];
+      }
+      s_need = need - cum;
+      s_prefix = prefix | ((uint32_t)bin << shift);
+    }
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t theta = s_prefix;   // key of the k-th largest score
+  const int need_eq = s_need;        // how many blocks with exactly that key to keep (lowest indices)
+
+  // ordered compaction: each thread owns a contiguous index range
+  const int per = (n_cand + kSelThreads - 1) / kSelThreads;
+  const int lo = min(tid * per, n_cand), hi = min(lo + per, n_cand);
+  int n_eq = 0;
+  for (int b = lo; b < hi; ++b) n_eq += (__float_as_uint(score[b]) == theta);
+  counts[tid] = n_eq;
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int i = 0; i < kSelThreads; ++i) { eq_base[i] = run; run += counts[i]; }
+  }
+  __syncthreads();
+  int eq_rank = eq_base[tid];
+  int n_keep = 0;
+  for (int b = lo; b < hi; ++b) {
+    uint32_t key = __float_as_uint(score[b]);
+    if (key > theta) ++n_keep;
+    else if (key == theta) { if (eq_rank < need_eq) ++n_keep; ++eq_rank; }
+  }
+  counts[tid] = n_keep;
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int i = 0; i < kSelThreads; ++i) { int c = counts[i]; counts[i] = run; run += c; }
+  }
+  __syncthreads();
+  int pos = counts[tid];
+  eq_rank = eq_base[tid];
+  for (int b = lo; b < hi; ++b) {
+    uint32_t key = __float_as_uint(score[b]);
+    bool keep = false;
+    if (key > theta) keep = true;
+    else if (key == theta) { keep = eq_rank < need_eq; ++eq_rank; }
+    if (keep && pos < k) out[pos++] = b;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host launchers
+// ------------------------------------------------------------------------------------------------
+template <int G>
+static cudaError_t launch_score_g(const Params &p, cudaStream_t stream) {
+  const int blocks_per_cta = 32;
+  dim3 grid((p.NB + blocks_per_cta - 1) / blocks_per_cta, p.B * p.Hkv);
+  size_t smem = (size_t)G * (p.D + p.Ds_pad) * sizeof(float);
+  switch (p.summ_dtype) {
+    case COBS_SUMM_FP32: score_generic_kernel<G, COBS_SUMM_FP32><<<grid, 256, smem, stream>>>(p, blocks_per_cta); break;
+    case COBS_SUMM_BF16: score_generic_kernel<G, COBS_SUMM_BF16><<<grid, 256, smem, stream>>>(p, blocks_per_cta); break;
+    default: score_generic_kernel<G, COBS_SUMM_FP4_E2M1><<<grid, 256, smem, stream>>>(p, blocks_per_cta); break;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_score(const Params &p, cudaStream_t stream) {
+  switch (p.G) {
+    case 1: return launch_score_g<1>(p, stream);
+    case 2: return launch_score_g<2>(p, stream);
+    case 4: return launch_score_g<4>(p, stream);
+    default: return launch_score_g<8>(p, stream);
+  }
+}
+
+cudaError_t launch_select(const Params &p, cudaStream_t stream) {
+  size_t smem = (size_t)p.NB * sizeof(float);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  select_kernel<<<p.B * p.Hkv, kSelThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace cobs

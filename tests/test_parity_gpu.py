@@ -1,0 +1,361 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Summaries for the score/select/attend checks are built by the oracle and uploaded
+bit for bit, so selection can be compared exactly (up to the tie band) and outputs within 2e-3.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cobs_oracle as O
+from paper_2607_09052_b200 import synth
+from parity import (OUT_TOL, SCORE_TOL, check_selection, oracle_attend, oracle_unit_step, oracle_unit_summaries,
+                    out_rel_err, upload_unit_summaries)
+
+pytestmark = pytest.mark.gpu
+
+WL = synth.named_workloads()
+
+
+def _binding():
+    from paper_2607_09052_b200 import binding
+    return binding
+
+
+def to_dev(inp):
+    return {k: (v.cuda() if isinstance(v, torch.Tensor) and k != "planted" else v) for k, v in inp.items()}
+
+
+def run_stage_s(wl, inp_cpu=None, units=None, inp_dev=None, summ=None):
+    """Score/select/attend parity for the given units (all by default). Returns a small report."""
+    B = _binding()
+    if inp_dev is None:
+        inp_cpu = synth.generate(wl) if inp_cpu is None else inp_cpu
+        inp_dev = to_dev(inp_cpu)
+    src = inp_dev if inp_cpu is None else inp_cpu
+    cfg = B.make_config(wl)
+    kv = B.make_kv(inp_dev)
+    if summ is None:
+        summ = B.SummaryBuffers(cfg, "cuda", inp_dev.get("u_q"))
+    ws = B.alloc_workspace(cfg, "cuda")
+    nb, hq, hkv, G, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.group, wl.head_dim
+    if units is None:
+        units = [(b, h) for b in range(nb) for h in range(hkv)]
+    ref = {}
+    for (b, h) in units:
+        st = oracle_unit_summaries(wl, src, b, h)
+        upload_unit_summaries(B, cfg, summ, b, h, st)
+        ref[(b, h)] = oracle_unit_step(wl, src, b, h, st)
+
+    sel_idx = torch.full((nb, hkv, wl.topk), -7, dtype=torch.int32, device="cuda")
+    sel_cnt = torch.full((nb, hkv), -7, dtype=torch.int32, device="cuda")
+    scores = torch.zeros((nb, hkv, wl.max_blocks), dtype=torch.float32, device="cuda")
+    B.cobs_score_select(cfg, inp_dev["q"], summ, inp_dev["seq_lens"], sel_idx, sel_cnt, scores, ws)
+
+    # attention on the ORACLE's selection, so a tie swap can neither hide nor fake an output error
+    sel_ref = torch.full((nb, hkv, wl.topk), -1, dtype=torch.int32)
+    cnt_ref = torch.zeros((nb, hkv), dtype=torch.int32)
+    for (b, h), r in ref.items():
+        sel_ref[b, h, :len(r["sel"])] = torch.from_numpy(r["sel"]).int()
+        cnt_ref[b, h] = len(r["sel"])
+    out_a = torch.zeros((nb, hq, D), dtype=torch.float32, device="cuda")
+    lse_a = torch.zeros((nb, hq), dtype=torch.float32, device="cuda")
+    B.cobs_sparse_decode(cfg, inp_dev["q"], kv, sel_ref.cuda(), cnt_ref.cuda(), out_a, lse_a, ws)
+
+    out_f = torch.zeros_like(out_a)
+    lse_f = torch.zeros_like(lse_a)
+    sel_f = torch.full_like(sel_idx, -7)
+    cnt_f = torch.full_like(sel_cnt, -7)
+    B.cobs_decode_step(cfg, inp_dev["q"], kv, summ, out_f, lse_f, sel_f, cnt_f, ws)
+    assert B.cobs_read_status(ws) == 0
+    torch.cuda.synchronize()
+
+    sel_idx, sel_cnt, scores = sel_idx.cpu(), sel_cnt.cpu(), scores.cpu().double().numpy()
+    out_a, lse_a, out_f, lse_f = out_a.cpu().numpy(), lse_a.cpu().numpy(), out_f.cpu().numpy(), lse_f.cpu().numpy()
+    sel_f, cnt_f = sel_f.cpu(), cnt_f.cpu()
+    report = {"swaps": 0, "max_score_err": 0.0, "max_out_err": 0.0}
+    for (b, h), r in ref.items():
+        T = int(src["seq_lens"][b])
+        n_sum = T // wl.block_size
+        n_cand = O.window_start(T, wl.window, wl.block_size) // wl.block_size
+        if n_sum:
+            err = np.max(np.abs(scores[b, h, :n_sum] - r["score"]) / np.maximum(r["score"], 1e-30))
+            report["max_score_err"] = max(report["max_score_err"], float(err))
+            assert err <= SCORE_TOL, (b, h, err)
+        ok, msg, exact = check_selection(sel_idx[b, h].tolist(), r["score"], n_cand, wl.topk)
+        assert ok, (b, h, msg)
+        assert int(sel_cnt[b, h]) == min(wl.topk, n_cand)
+        assert all(int(x) == -1 for x in sel_idx[b, h, int(sel_cnt[b, h]):])
+        report["swaps"] += 0 if exact else 1
+        # fused step: same selection bits as the two-call path
+        assert torch.equal(sel_f[b, h], sel_idx[b, h]) and int(cnt_f[b, h]) == int(sel_cnt[b, h])
+        hs = slice(h * G, (h + 1) * G)
+        ea = out_rel_err(out_a[b, hs], r["out"])
+        assert np.all(ea <= OUT_TOL), (b, h, ea)
+        assert np.allclose(lse_a[b, hs], r["lse"], atol=2e-3, rtol=0)
+        if exact:
+            ref_out, ref_lse = r["out"], r["lse"]
+        else:
+            ref_out, ref_lse = oracle_attend(wl, src, b, h, [int(x) for x in sel_f[b, h] if x >= 0])
+        ef = out_rel_err(out_f[b, hs], ref_out)
+        assert np.all(ef <= OUT_TOL), (b, h, ef)
+        assert np.allclose(lse_f[b, hs], ref_lse, atol=2e-3, rtol=0)
+        report["max_out_err"] = max(report["max_out_err"], float(ea.max()), float(ef.max()))
+    return report
+
+
+# --- the named workloads -------------------------------------------------------------------------------
+
+def test_cfg1_tiny_all_entry_points():
+    rep = run_stage_s(WL["cfg1_tiny"])
+    assert rep["swaps"] == 0
+
+
+def test_cfg2_32k_full():
+    run_stage_s(WL["cfg2_32k"])
+
+
+def test_cfg3a_subspace_fp4():
+    run_stage_s(WL["cfg3a_32k_subspace"].replace(batch=2))
+
+
+def test_cfg3b_k85_fp4():
+    run_stage_s(WL["cfg3b_32k_k85"].replace(batch=2), units=[(0, 0), (0, 5), (1, 3), (1, 7)])
+
+
+def test_cfg4_reduced_paged_rank8():
+    wl = WL["cfg4_128k"].replace(batch=2, seq_len=16384)
+    run_stage_s(wl)
+
+
+def test_cfg5_reduced_g8_block128():
+    wl = WL["cfg5_64k_g8"].replace(batch=2, seq_len=8192)
+    run_stage_s(wl)
+
+
+def test_cfg4_full_size_sampled_units():
+    """Full 128k x 16 workload in the launch configuration the benchmark times: inputs drawn on the
+    device, summaries built on the device for every block, then the sampled units' summaries replaced
+    by the oracle's so that their selection can be compared exactly."""
+    B = _binding()
+    wl = WL["cfg4_128k"]
+    inp = synth.generate(wl, "cuda")
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    B.cobs_build_summaries(cfg, B.make_kv(inp), 0, wl.max_blocks, summ, ws)
+    assert B.cobs_read_status(ws) == 0
+    run_stage_s(wl, inp_dev=inp, units=[(0, 0), (7, 3), (15, 7)], summ=summ)
+
+
+# --- shapes and edge cases ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("summary_dtype,scale_dtype", [("fp32", "fp32"), ("bf16", "fp32"), ("fp4", "fp32"),
+                                                       ("fp4", "fp16")])
+@pytest.mark.parametrize("G,D,L,P", [(1, 64, 32, 16), (2, 128, 64, 32), (4, 64, 128, 16), (8, 128, 16, 16)])
+def test_shape_grid(summary_dtype, scale_dtype, G, D, L, P):
+    wl = synth.Workload("grid", 2, 2 * G, 2, D, 40 * L, L, P, rank=3, topk=5, window=2 * L + 7,
+                        summary_dtype=summary_dtype, scale_dtype=scale_dtype, key_model="block_offset",
+                        planted=2, shuffle_pages=True, seed=11)
+    run_stage_s(wl)
+
+
+def test_ragged_lengths_and_degenerate_cases():
+    L = 64
+    # T < L (no summarised block), T inside the window only, partial last block, k larger than candidates
+    lens = [37, 200, 64 * 9 + 13, 64 * 30, 1]
+    wl = synth.Workload("ragged", len(lens), 8, 2, 128, 64 * 30, L, 16, rank=4, topk=12, window=130,
+                        summary_dtype="bf16", key_model="block_offset", planted=1, shuffle_pages=True, seed=12,
+                        seq_lens=lens)
+    run_stage_s(wl)
+
+
+def test_rank_zero_is_first_order_mean_pool():
+    wl = WL["cfg1_tiny"].replace(rank=0, summary_dtype="bf16")
+    run_stage_s(wl)
+
+
+def test_subspace_odd_dimension_bf16_and_fp32():
+    for dt in ("bf16", "fp32"):
+        wl = synth.Workload("sub", 1, 8, 2, 128, 64 * 24, 64, 64, rank=4, topk=6, window=128, summary_dtype=dt,
+                            sub_dim=53, key_model="block_offset", query_model="spectrum", planted=2, seed=13)
+        run_stage_s(wl)
+
+
+def test_invalid_selection_is_reported_not_faulted():
+    """An out-of-range block index is skipped by the kernel and surfaces as a status code."""
+    B = _binding()
+    wl = WL["cfg1_tiny"]
+    inp = to_dev(synth.generate(wl))
+    cfg = B.make_config(wl)
+    ws = B.alloc_workspace(cfg, "cuda")
+    sel = torch.tensor([[[0, 5, 31, 99]]], dtype=torch.int32, device="cuda")   # 31 lies in the window, 99 is outside
+    cnt = torch.tensor([[4]], dtype=torch.int32, device="cuda")
+    out = torch.zeros((1, 4, 64), dtype=torch.float32, device="cuda")
+    B.cobs_sparse_decode(cfg, inp["q"], B.make_kv(inp), sel, cnt, out, None, ws)
+    assert B.cobs_read_status(ws) == 6
+    B.cobs_reset_status(ws)
+    assert B.cobs_read_status(ws) == 0
+    # the valid part of the request was still served: equals the oracle on blocks {0, 5}
+    cpu = synth.generate(wl)
+    o_ref, _ = oracle_attend(wl, cpu, 0, 0, [0, 5])
+    assert np.all(out_rel_err(out[0].cpu().numpy(), o_ref) <= OUT_TOL)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    B = _binding()
+    wl = WL["cfg2_32k"].replace(seq_len=4096)
+    cpu = synth.generate(wl)
+    inp = to_dev(cpu)
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    kv = B.make_kv(inp)
+    B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, summ, ws)
+    out_d = torch.zeros((1, 32, 128), dtype=torch.float32, device="cuda")
+    sel_d = torch.zeros((1, 8, wl.topk), dtype=torch.int32, device="cuda")
+    cnt_d = torch.zeros((1, 8), dtype=torch.int32, device="cuda")
+    B.cobs_decode_step(cfg, inp["q"], kv, summ, out_d, None, sel_d, cnt_d, ws)
+    q_h = cpu["q"].pin_memory()
+    out_h = torch.zeros((1, 32, 128), dtype=torch.float32).pin_memory()
+    sel_h = torch.zeros((1, 8, wl.topk), dtype=torch.int32).pin_memory()
+    cnt_h = torch.zeros((1, 8), dtype=torch.int32).pin_memory()
+    B.cobs_decode_step_host(cfg, q_h, kv, summ, out_h, sel_h, cnt_h, ws)
+    assert torch.equal(out_h, out_d.cpu()) and torch.equal(sel_h, sel_d.cpu()) and torch.equal(cnt_h, cnt_d.cpu())
+
+
+# --- quantiser (bit exact) -----------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("scale_dtype", ["fp32", "fp16"])
+@pytest.mark.parametrize("ds", [128, 85, 64])
+def test_quantiser_bit_exact(scale_dtype, ds):
+    B = _binding()
+    wl = WL["cfg4_128k"].replace(sub_dim=0 if ds == 128 else ds, scale_dtype=scale_dtype, rank=4)
+    cfg = B.make_config(wl)
+    r = np.random.default_rng(ds)
+    n = 4 * 300
+    xi = (r.normal(size=(n, ds)) * np.exp(r.normal(size=(n, 1)) * 2)).astype(np.float32)
+    grid = np.array([6, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, -0.25, -2.5, 0.0, -0.0, 5.999, 0.2499, 6.0], np.float32)
+    xi[0, :len(grid)] = grid; xi[0, len(grid):] = 0
+    xi[1] = 0.0
+    xi[2] = 1e-30
+    xi[3, :] = np.linspace(-6, 6, ds)
+    codes_ref, scale_ref = O.quantise_e2m1(xi, scale_dtype)
+    ds_pad = B.cobs_padded_sub_dim(cfg)
+    codes = torch.full((n, ds_pad // 2), 0xEE, dtype=torch.uint8, device="cuda")
+    scale = torch.zeros(n, dtype=torch.float16 if scale_dtype == "fp16" else torch.float32, device="cuda")
+    B.cobs_quantise_xi(cfg, torch.from_numpy(xi).cuda(), codes, scale)
+    got = B.unpack_fp4_rows(codes, ds_pad).cpu().numpy()
+    assert np.array_equal(got[:, :ds], codes_ref)
+    assert np.all(got[:, ds:] == 0)
+    assert np.array_equal(scale.float().cpu().numpy(), scale_ref)
+
+
+# --- builder (backward error; eigenvectors of close eigenvalues are not unique to rounding) ---------------------
+
+def check_builder(wl, units):
+    B = _binding()
+    cpu = synth.generate(wl)
+    inp = to_dev(cpu)
+    cfg32 = B.make_config(wl.replace(summary_dtype="fp32"))
+    s32 = B.SummaryBuffers(cfg32, "cuda", inp.get("u_q"))
+    ws = B.alloc_workspace(cfg32, "cuda")
+    kv = B.make_kv(inp)
+    B.cobs_build_summaries(cfg32, kv, 0, wl.max_blocks, s32, ws)
+    assert B.cobs_read_status(ws) == 0
+    mean32, xi32, _ = B.summary_views(cfg32, s32)
+    # determinism: a second build gives the same bits
+    s32b = B.SummaryBuffers(cfg32, "cuda", inp.get("u_q"))
+    B.cobs_build_summaries(cfg32, kv, 0, wl.max_blocks, s32b, ws)
+    assert torch.equal(s32.xi, s32b.xi) and torch.equal(s32.mean, s32b.mean)
+
+    r, L = wl.rank, wl.block_size
+    for (b, h) in units:
+        K, _ = synth.unit_kv(cpu, wl, b, h)
+        K = K.numpy()
+        u_q = cpu["u_q"][h].double().numpy() if wl.sub_dim else None
+        q = synth.unit_q(cpu, wl, b, h).numpy()
+        qt = O.scale_query(q) if u_q is None else O.scale_query(q) @ u_q
+        n_sum = int(cpu["seq_lens"][b]) // L
+        xi_g = xi32[b, h, :n_sum].double().cpu().numpy()
+        mean_g = mean32[b, h, :n_sum].double().cpu().numpy()
+        for blk in range(n_sum):
+            kb = K[blk * L:(blk + 1) * L]
+            kbar, sigma = O.block_mean_and_covariance(kb)
+            if u_q is not None:
+                sigma = u_q.T @ sigma @ u_q
+            lam = np.sort(np.linalg.eigvalsh(sigma))[::-1]
+            lam0 = lam[0]
+            assert np.max(np.abs(mean_g[blk] - kbar)) <= 1e-6 * max(1.0, np.max(np.abs(kbar)))
+            x = xi_g[blk]
+            for i in range(r):
+                n2 = x[i] @ x[i]
+                assert abs(n2 - lam[i]) <= 2e-5 * lam0, (b, h, blk, i, n2, lam[i])
+                resid = np.linalg.norm(sigma @ x[i] - n2 * x[i])
+                assert resid <= 1e-4 * lam0 * np.sqrt(n2), (b, h, blk, i, resid)
+                j = int(np.argmax(np.abs(x[i])))
+                assert x[i, j] > 0
+                for k2 in range(i):
+                    assert abs(x[i] @ x[k2]) <= 1e-4 * np.sqrt(n2 * (x[k2] @ x[k2]))
+            # the quadratic form the scorer will see
+            for g in range(q.shape[0]):
+                got = sum((x[i] @ qt[g]) ** 2 for i in range(r))
+                _, xr, _ = O.scaled_eigenvectors_gram(kb, r, u_q)
+                want = sum((xr[i] @ qt[g]) ** 2 for i in range(r))
+                slack = 1e-4 * lam0 * (qt[g] @ qt[g]) + (lam[r - 1] - lam[r] if (lam[r - 1] - lam[r]) < 1e-3 * lam0 else 0) * (qt[g] @ qt[g])
+                assert abs(got - want) <= slack, (b, h, blk, g, got, want)
+
+    # storage formats: the device's bf16 / FP4 outputs are its own fp32 factors pushed through the
+    # storage rounding (bf16: RNE; FP4: the quantiser, itself bit-exact against the oracle elsewhere)
+    if wl.summary_dtype != "fp32":
+        cfg = B.make_config(wl)
+        s = B.SummaryBuffers(cfg, "cuda", inp.get("u_q"))
+        B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, s, ws)
+        mean_s, xi_s, scale_s = B.summary_views(cfg, s)
+        assert torch.equal(mean_s, mean32.to(torch.bfloat16))
+        if wl.summary_dtype == "bf16":
+            assert torch.equal(xi_s, xi32.to(torch.bfloat16))
+        else:
+            ds = wl.sub_dim or wl.head_dim
+            flat = xi32.reshape(-1, ds).contiguous()
+            codes = torch.zeros((flat.shape[0], xi_s.shape[-1]), dtype=torch.uint8, device="cuda")
+            scale = torch.zeros(flat.shape[0], dtype=scale_s.dtype, device="cuda")
+            B.cobs_quantise_xi(cfg, flat, codes, scale)
+            assert torch.equal(codes.view_as(xi_s), xi_s) and torch.equal(scale.view_as(scale_s), scale_s)
+            # and against the oracle's quantiser applied to the oracle's own factors: informational agreement
+    assert B.cobs_read_status(ws) == 0
+
+
+def test_builder_cfg1_fp32():
+    check_builder(WL["cfg1_tiny"], [(0, 0)])
+
+
+def test_builder_cfg2_like_bf16():
+    check_builder(WL["cfg2_32k"].replace(seq_len=4096), [(0, 0), (0, 7)])
+
+
+def test_builder_cfg4_like_fp4_paged():
+    check_builder(WL["cfg4_128k"].replace(batch=2, seq_len=4096), [(0, 1), (1, 6)])
+
+
+def test_builder_cfg3a_like_subspace():
+    check_builder(WL["cfg3a_32k_subspace"].replace(batch=1, seq_len=2048), [(0, 2)])
+
+
+def test_builder_cfg5_like_block128():
+    check_builder(WL["cfg5_64k_g8"].replace(batch=1, seq_len=4096), [(0, 4)])
+
+
+def test_builder_constant_key_block_gives_zero_factors():
+    B = _binding()
+    wl = WL["cfg1_tiny"].replace(summary_dtype="fp4")
+    inp = to_dev(synth.generate(wl))
+    inp["k_pages"][3] = inp["k_pages"][3, :, :1, :]          # every key of block 3 equal
+    cfg = B.make_config(wl)
+    s = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    B.cobs_build_summaries(cfg, B.make_kv(inp), 0, wl.max_blocks, s, ws)
+    mean, xi, scale = B.summary_views(cfg, s)
+    assert torch.all(xi[0, 0, 3] == 0) and torch.all(scale[0, 0, 3] == 0)
+    assert torch.equal(mean[0, 0, 3], inp["k_pages"][3, 0, 0])
+    assert torch.any(xi[0, 0, 2] != 0)
