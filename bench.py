@@ -1,0 +1,386 @@
+"""Benchmark of the fused COBS decode step (cobs_decode_step) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one pass of the whole per-decode-step path (block scoring from the summaries, top-k
+selection, block-sparse attention over the selected blocks plus the window) over one batch of a
+synthetic long-context workload whose KV cache and summaries are resident in HBM.  The reported
+value is the whole-job achieved HBM bandwidth: algorithmic bytes per step (summary records of every
+summarised block + K and V of the selected and window blocks + q + out) times the number of ranks,
+divided by the step time (CUDA events, max over ranks).  Prints ONE JSON line on rank 0.
+
+With N > 1 (launched by torch.distributed.run) every rank holds its own batch of sequences: the path
+shards over (sequence, KV head) with no collective, so scaling is weak.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2607_09052_b200 import synth  # noqa: E402
+
+DEFAULT_WORKLOAD = "cfg4_128k"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def algorithmic_bytes(wl: synth.Workload, record_bytes: int) -> int:
+    """Bytes one step must read or write: summary records of every summarised block, K and V of the
+    selected and window blocks, q, out, the page-table entries of the blocks read, and U_Q."""
+    total = 0
+    L, D = wl.block_size, wl.head_dim
+    for t in wl.lens():
+        n_sum = t // L
+        ws = (max(0, t - wl.window) // L) * L
+        n_cand = ws // L
+        n_sel = min(wl.topk, n_cand)
+        kv_tokens = n_sel * L + (t - ws)
+        total += wl.n_kv_heads * (n_sum * record_bytes + kv_tokens * D * 2 * 2)
+        total += (kv_tokens + wl.page_size - 1) // wl.page_size * 4
+    total += wl.batch * wl.n_q_heads * D * (2 + 4)
+    if wl.sub_dim:
+        total += wl.n_kv_heads * D * wl.sub_dim * 4
+    return total
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def run_ours(args):
+    from paper_2607_09052_b200 import binding as B
+    from paper_2607_09052_b200 import build as build_mod
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if rank == 0:
+        build_mod.build()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    B.lib()
+
+    wl = synth.named_workloads()[args.workload]
+    wl = wl.replace(seed=wl.seed + 1000 * rank)        # every rank draws its own sequences
+    dev = torch.device("cuda", local_rank)
+    inp = synth.generate(wl, dev)
+    cfg = B.make_config(wl)
+    kv = B.make_kv(inp)
+    summ = B.SummaryBuffers(cfg, dev, inp.get("u_q"))
+    ws = B.alloc_workspace(cfg, dev)
+    stream = torch.cuda.current_stream()
+
+    # summaries of every block, built by the library (set-up, timed separately)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, summ, ws)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    build_ms = ev0.elapsed_time(ev1)
+    if B.cobs_read_status(ws) != 0:
+        raise RuntimeError("device status after build_summaries")
+
+    nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+    out = torch.zeros((nb, hq, D), dtype=torch.float32, device=dev)
+    sel = torch.zeros((nb, hkv, wl.topk), dtype=torch.int32, device=dev)
+    cnt = torch.zeros((nb, hkv), dtype=torch.int32, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    mb, xb, sb = B.cobs_summary_bytes(cfg)
+    record = (mb + xb + sb) // (nb * hkv * wl.max_blocks)
+    step_bytes = algorithmic_bytes(wl, record)
+
+    def step():
+        B.cobs_decode_step(cfg, inp["q"], kv, summ, out, None, sel, cnt, ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+
+    # ---- timed region: exactly K steps, an L2 flush (not timed) before each ----------------------------
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    launches0 = B.cobs_kernel_launches()
+    t_wall0 = time.perf_counter()
+    for i in range(args.steps):
+        flush.zero_()
+        starts[i].record(stream)
+        step()
+        ends[i].record(stream)
+    barrier()
+    wall_s = time.perf_counter() - t_wall0
+    launches = B.cobs_kernel_launches() - launches0
+    clocks = sampler.stop() if sampler else None
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    total_ms = sum(step_ms)
+    if B.cobs_read_status(ws) != 0:
+        raise RuntimeError("device status after the timed steps")
+
+    # ---- dominant kernels on their own, same launch configuration (for the roofline line) --------------
+    def time_call(fn, n):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b_ in evs:
+            flush.zero_()
+            a.record(stream)
+            fn()
+            b_.record(stream)
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b_) for a, b_ in evs) / n
+
+    n_sub = max(3, min(args.steps, 20))
+    score_ms = time_call(lambda: B.cobs_score_select(cfg, inp["q"], summ, inp["seq_lens"], sel, cnt, None, ws), n_sub)
+    attend_ms = time_call(lambda: B.cobs_sparse_decode(cfg, inp["q"], kv, sel, cnt, out, None, ws), n_sub)
+    summary_bytes = sum(hkv * (t // wl.block_size) * record for t in wl.lens())
+    kv_bytes = step_bytes - summary_bytes
+
+    # ---- end to end through the host-buffer entry point ------------------------------------------------
+    q_host = inp["q"].cpu().pin_memory()
+    out_host = torch.zeros((nb, hq, D), dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        B.cobs_decode_step_host(cfg, q_host, kv, summ, out_host, None, None, ws)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+        B.cobs_decode_step_host(cfg, q_host, kv, summ, out_host, None, None, ws)
+    e2e_s = time.perf_counter() - t0
+    # the flush and its synchronise are inside this wall-clock loop; time them alone and take them out
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+    e2e_s = max(e2e_s - (time.perf_counter() - t0), 1e-9)
+
+    t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_s = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = read_peaks()
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    dominant = ("sparse_decode(attend+combine)", kv_bytes, attend_ms) if attend_ms >= score_ms else \
+               ("score_select(score+select)", summary_bytes, score_ms)
+    achieved = dominant[1] / (dominant[2] * 1e-3) / 1e9
+    line = {
+        "metric": "fused COBS decode step: achieved HBM GB/s (algorithmic bytes per step / step time)",
+        "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(ms_per_step, 6), "us_per_step": round(ms_per_step * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "batch_per_gpu": nb, "global_batch": nb * world, "context": wl.seq_len,
+                   "n_q_heads": hq, "n_kv_heads": hkv, "head_dim": D, "block_size": wl.block_size,
+                   "page_size": wl.page_size, "topk": wl.topk, "window": wl.window, "rank": wl.rank,
+                   "sub_dim": wl.sub_dim, "summary_dtype": wl.summary_dtype, "scale_dtype": wl.scale_dtype,
+                   "record_bytes": record, "algorithmic_bytes_per_step": step_bytes,
+                   "l2": f"{L2_FLUSH_BYTES >> 20} MiB write between timed steps (outside the events); "
+                         f"step traffic {step_bytes / 2**20:.1f} MiB",
+                   "sharding": "independent sequences per rank, no collective"},
+        "frac_of_measured_peak": round(value / (world * peak), 4), "peak_gbs": peak, "peak_kind": peak_kind,
+        "frac_of_nominal_8tbs": round(value / (world * 8000.0), 4),
+        "roofline": {"bound": "hbm", "kernel": dominant[0], "achieved": round(achieved, 2), "peak": peak,
+                     "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": None,
+                     "algorithmic_bytes": dominant[1], "launch_ms": round(dominant[2], 6),
+                     "note": f"of {peak_kind}; score_select {score_ms * 1e3:.1f} us for {summary_bytes} B, "
+                             f"sparse_decode {attend_ms * 1e3:.1f} us for {kv_bytes} B, timed alone after the steps"},
+        "e2e": {"value": round(world * step_bytes / (e2e_s / args.steps) / 1e9, 2), "unit": "GB/s",
+                "us_per_step": round(e2e_s / args.steps * 1e6, 2),
+                "h2d_bytes_per_step": q_host.numel() * 2, "d2h_bytes_per_step": out_host.numel() * 4},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "build_summaries_ms": round(build_ms, 3),
+        "wall_s_timed_region": round(wall_s, 4),
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(wl, record, budget_s=12.0)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------------------------
+# CPU baseline / reference arm: the oracle as it stands, on the host cores, on a bounded sample.
+# ----------------------------------------------------------------------------------------------------------
+
+def oracle_sample(wl: synth.Workload, n_units: int):
+    """Inputs and oracle-built summaries for the first n_units (sequence 0, KV heads 0..) of a workload
+    reduced to one sequence (same shapes per unit as the full workload)."""
+    from oracle import cobs_oracle as O
+    small = wl.replace(batch=1, seq_lens=None)
+    inp = synth.generate(small, "cpu")
+    units = []
+    for h in range(min(n_units, small.n_kv_heads)):
+        K, V = synth.unit_kv(inp, small, 0, h)
+        q = synth.unit_q(inp, small, 0, h).numpy()
+        u_q = inp["u_q"][h].double().numpy() if small.sub_dim else None
+        mean, xi, _ = O.build_summaries(K.numpy(), small.block_size, small.rank, u_q)
+        st = O.store_summaries(mean, xi, small.summary_dtype, small.scale_dtype)
+        units.append((q, K.numpy(), V.numpy(), st, u_q))
+    return small, units
+
+
+def oracle_time_steps(small, units, repeats: int):
+    from oracle import cobs_oracle as O
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        for q, K, V, st, u_q in units:
+            O.decode_step(q, K, V, small.seq_len, st, small.block_size, small.topk, small.window, u_q)
+    return time.perf_counter() - t0
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(wl, record, budget_s: float):
+    n_units = 2
+    small, units = oracle_sample(wl, n_units)
+    one = oracle_time_steps(small, units, 1)
+    repeats = max(1, min(200, int(budget_s / max(one, 1e-6))))
+    elapsed = oracle_time_steps(small, units, repeats)
+    unit_bytes = algorithmic_bytes(small, record) / small.n_kv_heads
+    gbs = repeats * len(units) * unit_bytes / elapsed / 1e9
+    return {"value": round(gbs, 4), "unit": "GB/s", "cores": host_threads(), "kind": "oracle",
+            "sample": f"{len(units)} (sequence, KV head) units of {wl.name} x {repeats} repeats, "
+                      f"score + select + attend per unit (summaries prebuilt), {elapsed:.1f} s",
+            "us_per_step_extrapolated": round(elapsed / (repeats * len(units)) * wl.batch * wl.n_kv_heads * 1e6, 1)}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    wl = synth.named_workloads()[args.workload]
+    mb = wl.head_dim * (4 if wl.summary_dtype == "fp32" else 2)
+    ds = wl.sub_dim or wl.head_dim
+    if wl.summary_dtype == "fp4":
+        pad = (ds + 7) // 8 * 8
+        while wl.rank and (wl.rank * pad // 2) % 16:
+            pad += 8
+        record = mb + wl.rank * pad // 2 + wl.rank * (2 if wl.scale_dtype == "fp16" else 4)
+    else:
+        record = mb + wl.rank * ds * (4 if wl.summary_dtype == "fp32" else 2)
+    small, units = oracle_sample(wl, 2)
+    for _ in range(args.warmup):
+        oracle_time_steps(small, units, 1)
+    times = [oracle_time_steps(small, units, 1) for _ in range(args.steps)]
+    per_step_s = sum(times) / len(times)
+    unit_bytes = algorithmic_bytes(small, record) / small.n_kv_heads
+    gbs = len(units) * unit_bytes / per_step_s / 1e9
+    sample = f"each step = {len(units)} (sequence, KV head) units of {wl.name} (of {wl.batch * wl.n_kv_heads}), " \
+             f"score + select + attend by the CPU oracle, summaries prebuilt"
+    line = {"impl": "reference",
+            "metric": "fused COBS decode step: achieved HBM GB/s (algorithmic bytes per step / step time)",
+            "value": round(gbs, 4), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(per_step_s * 1e3, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "context": wl.seq_len, "sample": sample},
+            "cpu_baseline": {"value": round(gbs, 4), "unit": "GB/s", "kind": "oracle", "cores": host_threads(),
+                             "sample": sample},
+            "e2e": {"value": round(gbs, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.named_workloads()))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -198,6 +198,10 @@ int32_t cobs_decode_step_host(const cobs_config *cfg, const void *q_host, const 
                               const cobs_summaries *summ, float *out_host, int32_t *sel_idx_host_or_null,
                               int32_t *sel_cnt_host_or_null, void *workspace, size_t workspace_bytes, void *stream);
 
+/* Number of kernels this library has launched in this process so far (host-side counter; the paper
+ * has no counterpart: it exists so that a benchmark can state how many launches a timed region held). */
+int64_t cobs_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,7 @@ SCALE_DTYPES = {"fp32": 0, "fp16": 1}
 EXPORTS = [
     "cobs_status_string", "cobs_padded_sub_dim", "cobs_summary_bytes", "cobs_workspace_bytes", "cobs_reset_status",
     "cobs_read_status", "cobs_build_summaries", "cobs_quantise_xi", "cobs_score_select", "cobs_sparse_decode",
-    "cobs_decode_step", "cobs_decode_step_host",
+    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches",
 ]
 
 
@@ -63,8 +63,13 @@ def lib():
         l.cobs_status_string.argtypes = [C.c_int32]
         for name in EXPORTS[1:]:
             getattr(l, name).restype = C.c_int32
+        l.cobs_kernel_launches.restype = C.c_int64
         _lib = l
     return _lib
+
+
+def cobs_kernel_launches() -> int:
+    return int(lib().cobs_kernel_launches())
 
 
 def status_string(status: int) -> str:

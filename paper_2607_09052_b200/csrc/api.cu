@@ -4,7 +4,12 @@
 
 #include "common.cuh"
 
+#include <atomic>
+
 namespace cobs {
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_select(const Params &p, cudaStream_t stream);
 cudaError_t launch_attend(const Params &p, cudaStream_t stream);
@@ -144,6 +149,8 @@ const char *cobs_status_string(int32_t s) {
     default: return "unknown status";
   }
 }
+
+int64_t cobs_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t cobs_padded_sub_dim(const cobs_config *cfg) {
   if (validate_config(cfg) != COBS_OK) return -1;

@@ -39,6 +39,9 @@ struct Params {
   float *lse;                 // optional [B][Hq]
 };
 
+// host-side count of kernel launches (see cobs_kernel_launches)
+void count_launch(int n = 1);
+
 __device__ __forceinline__ void report(int32_t *status, int code) {
   if (status) atomicCAS(status, 0, code);
 }

@@ -247,6 +247,7 @@ static cudaError_t launch_score_g(const Params &p, cudaStream_t stream) {
     case COBS_SUMM_BF16: score_generic_kernel<G, COBS_SUMM_BF16><<<grid, 256, smem, stream>>>(p, blocks_per_cta); break;
     default: score_generic_kernel<G, COBS_SUMM_FP4_E2M1><<<grid, 256, smem, stream>>>(p, blocks_per_cta); break;
   }
+  count_launch();
   return cudaGetLastError();
 }
 
@@ -266,6 +267,7 @@ cudaError_t launch_select(const Params &p, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
   }
   select_kernel<<<p.B * p.Hkv, kSelThreads, smem, stream>>>(p);
+  count_launch();
   return cudaGetLastError();
 }
 

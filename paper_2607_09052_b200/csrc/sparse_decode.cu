@@ -198,6 +198,7 @@ static cudaError_t launch_attend_gd(const Params &p, cudaStream_t stream) {
   }
   dim3 grid(p.n_splits, p.B * p.Hkv);
   attend_kernel<G, D><<<grid, kAttThreads, smem, stream>>>(p);
+  count_launch();
   return cudaGetLastError();
 }
 
@@ -216,6 +217,7 @@ cudaError_t launch_attend(const Params &p, cudaStream_t stream) {
   }
   if (e != cudaSuccess) return e;
   combine_kernel<<<p.B * p.Hq, p.D, 0, stream>>>(p);
+  count_launch();
   return cudaGetLastError();
 }
 

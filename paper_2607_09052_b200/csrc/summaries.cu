@@ -334,6 +334,7 @@ cudaError_t launch_build(const Params &p, int block_begin, int block_end, cudaSt
   if (e != cudaSuccess) return e;
   const long long n_cta = (long long)p.B * p.Hkv * n_range;
   build_kernel<<<(unsigned)n_cta, kBuildThreads, smem, stream>>>(p, block_begin, block_end);
+  count_launch();
   return cudaGetLastError();
 }
 
@@ -343,6 +344,7 @@ cudaError_t launch_quantise(const float *xi, long long n_vectors, int Ds, int Ds
   const int wpb = 8;
   quantise_kernel<<<(unsigned)((n_vectors + wpb - 1) / wpb), wpb * 32, 0, stream>>>(xi, n_vectors, Ds, Ds_pad,
                                                                                  scale_dtype, (uint8_t *)codes, scale);
+  count_launch();
   return cudaGetLastError();
 }
 
