@@ -73,7 +73,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -164,13 +164,18 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    t_warm = time.perf_counter()
+    n_warm = 0
+    while n_warm < args.warmup or time.perf_counter() - t_warm < 0.6:   # >= W steps, and long enough for clock samples
         flush.zero_()
         step()
+        n_warm += 1
+        if n_warm % 16 == 0:
+            torch.cuda.synchronize()
     barrier()
 
     # ---- timed region: exactly K steps, an L2 flush (not timed) before each ----------------------------
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     launches0 = B.cobs_kernel_launches()
@@ -321,7 +326,7 @@ def cpu_baseline(wl, record, budget_s: float):
     n_units = 2
     small, units = oracle_sample(wl, n_units)
     one = oracle_time_steps(small, units, 1)
-    repeats = max(1, min(200, int(budget_s / max(one, 1e-6))))
+    repeats = max(1, min(5000, int(budget_s / max(one, 1e-6))))
     elapsed = oracle_time_steps(small, units, repeats)
     unit_bytes = algorithmic_bytes(small, record) / small.n_kv_heads
     gbs = repeats * len(units) * unit_bytes / elapsed / 1e9

@@ -112,8 +112,8 @@ typedef struct {
 
 const char *cobs_status_string(int32_t status);
 
-/* Row length in elements of a packed FP4 factor row: Ds rounded up so that every block's factor record
- * (r rows) is a whole number of 16-byte units and every row a whole number of 4-byte words. */
+/* Row length in elements of a packed FP4 factor row: Ds rounded up to a multiple of 32 codes, so that
+ * every row is a whole number of 16-byte units and starts on a 16-byte boundary. */
 int32_t cobs_padded_sub_dim(const cobs_config *cfg);
 
 /* Bytes of each summary array for cfg (scale_bytes = 0 unless FP4).  Host-only arithmetic. */

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcobs.so")
-SOURCES = ["api.cu", "score_select.cu", "sparse_decode.cu", "summaries.cu"]
+SOURCES = ["api.cu", "score_select.cu", "score_mma.cu", "sparse_decode.cu", "summaries.cu"]
 
 
 def nvcc_path() -> str:

@@ -21,12 +21,9 @@ size_t build_smem_bytes(const Params &p);
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-static int padded_sub_dim(int Ds, int r) {
-  int pad = (Ds + 7) / 8 * 8;
-  if (r > 0)
-    while (((size_t)r * pad / 2) % 16 != 0) pad += 8;
-  return pad;
-}
+// Packed FP4 rows are padded to a whole number of 16-byte units (32 codes), so that every row of
+// every block starts on a 16-byte boundary.
+static int padded_sub_dim(int Ds, int /*r*/) { return (Ds + 31) / 32 * 32; }
 
 static bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 

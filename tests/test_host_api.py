@@ -52,14 +52,13 @@ def test_summary_record_bytes_follow_the_papers_accounting():
     assert record_bytes(wl["cfg2_32k"]) == (1280, 1024)            # bf16 mean 256 + 4 x 128 x 2
     assert record_bytes(wl["cfg3b_32k_k85"]) == (528, 272)         # 256 + (4 x 64 + 4 x 4): the table's 272
     assert record_bytes(wl["cfg4_128k"]) == (800, 544)             # r = 8
-    assert record_bytes(wl["cfg3a_32k_subspace"]) == (448, 192)    # 85 -> 88 nibbles per row
+    assert record_bytes(wl["cfg3a_32k_subspace"]) == (464, 208)    # 85 -> 96 codes (48 B) per row
     assert record_bytes(wl["cfg4_128k"].replace(scale_dtype="fp16")) == (784, 528)
     # the factor bytes agree with the oracle's accounting wherever no padding is involved
     for r, d in ((4, 128), (4, 64), (6, 128)):
         w = wl["cfg3b_32k_k85"].replace(rank=r, sub_dim=0 if d == 128 else d)
-        if (r * d // 2) % 16 == 0:
-            assert record_bytes(w)[1] == O.factor_bytes(r, d, "fp4")
-    assert B.cobs_padded_sub_dim(B.make_config(wl["cfg3a_32k_subspace"])) == 88
+        assert record_bytes(w)[1] == O.factor_bytes(r, d, "fp4")
+    assert B.cobs_padded_sub_dim(B.make_config(wl["cfg3a_32k_subspace"])) == 96
 
 
 def test_workspace_size_and_alignment_rules():
@@ -110,7 +109,7 @@ def test_entry_points_reject_bad_pointers_before_launching():
 def test_pack_unpack_fp4_layout():
     import torch
     codes = torch.arange(16, dtype=torch.uint8).repeat(2)[:21].view(1, 21)
-    packed = B.pack_fp4_rows(codes, 24)
-    assert packed.shape == (1, 12)
+    packed = B.pack_fp4_rows(codes, 32)
+    assert packed.shape == (1, 16)
     assert packed[0, 0] == (0 | (1 << 4)) and packed[0, 10] == 4 and packed[0, 11] == 0
     assert torch.equal(B.unpack_fp4_rows(packed, 21), codes)
