@@ -167,7 +167,7 @@ def run_ours(args):
     sampler = ClockSampler(local_rank) if rank == 0 else None
     t_warm = time.perf_counter()
     n_warm = 0
-    while n_warm < args.warmup or time.perf_counter() - t_warm < 0.6:   # >= W steps, and long enough for clock samples
+    while n_warm < args.warmup or time.perf_counter() - t_warm < args.clock_warm_s:   # >= W steps, and long enough for clock samples
         flush.zero_()
         step()
         n_warm += 1
@@ -379,6 +379,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.named_workloads()))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--clock-warm-s", type=float, default=0.6,
+                    help="keep warming up at least this long so that the clock sampler has samples")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -109,13 +109,15 @@ __global__ void __launch_bounds__(kScoreThreads, 4) score_mma_kernel(Params p, i
         __syncthreads();
         for (int i = tid; i < G * p.Ds_pad; i += kScoreThreads) {
           const int g = i / p.Ds_pad, s = i - g * p.Ds_pad;
+          // full space: the raw bf16 query (exact in f16 after the power-of-two scaling below; the
+          // 1/sqrt(D) factor is applied to the tile result instead); subspace: q~ = U_Q^T q / sqrt(D)
           float v = 0.f;
           if (s < p.Ds) {
             if (p.u_q) {
               const float *uq = p.u_q + (size_t)h * D * p.Ds + s;
               for (int d = 0; d < D; ++d) v = fmaf(uq[(size_t)d * p.Ds], qs[g * D + d], v);
             } else {
-              v = qs[g * D + s];
+              v = __bfloat162float(qg[g * D + s]);
             }
           }
           qt[i] = v;
@@ -152,8 +154,9 @@ __global__ void __launch_bounds__(kScoreThreads, 4) score_mma_kernel(Params p, i
             bq[t][2 * j + 1][0] = pack_f16(hi[2], hi[6]); bq[t][2 * j + 1][1] = pack_f16(hi[3], hi[7]);
           }
         }
-        m0 = (2 * tig < G) ? mult[2 * tig] * kDecodeScale : 0.f;
-        m1 = (2 * tig + 1 < G) ? mult[2 * tig + 1] * kDecodeScale : 0.f;
+        const float post = p.u_q ? kDecodeScale : kDecodeScale * inv_sqrt_d;
+        m0 = (2 * tig < G) ? mult[2 * tig] * post : 0.f;
+        m1 = (2 * tig + 1 < G) ? mult[2 * tig + 1] * post : 0.f;
       }
     }
     const int base = chunk * kBlocksPerItem + warp * 16;
