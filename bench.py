@@ -125,6 +125,8 @@ def run_ours(args):
     B.lib()
 
     wl = synth.named_workloads()[args.workload]
+    if args.batch:
+        wl = wl.replace(batch=args.batch, name=f"{wl.name}[batch={args.batch}]")
     wl = wl.replace(seed=wl.seed + 1000 * rank)        # every rank draws its own sequences
     dev = torch.device("cuda", local_rank)
     inp = synth.generate(wl, dev)
@@ -379,6 +381,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.named_workloads()))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
     ap.add_argument("--clock-warm-s", type=float, default=0.6,
                     help="keep warming up at least this long so that the clock sampler has samples")
     args = ap.parse_args()

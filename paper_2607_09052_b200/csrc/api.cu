@@ -25,6 +25,12 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 // every block starts on a 16-byte boundary.
 static int padded_sub_dim(int Ds, int /*r*/) { return (Ds + 31) / 32 * 32; }
 
+constexpr int kMaxGroupsPerCta = 1024;   // 16-token groups one attention CTA can index
+
+static int max_items(const cobs_config *c) {
+  return c->topk + (c->window + c->block_size - 1) / c->block_size + 1;
+}
+
 static bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
 static int32_t validate_config(const cobs_config *c) {
@@ -47,13 +53,20 @@ static int32_t validate_config(const cobs_config *c) {
   if (c->max_pages_per_seq < 1) return COBS_ERR_INVALID_ARG;
   // the page table must cover every token a sequence may hold: NB * L + L - 1 at most
   if ((long long)c->max_pages_per_seq * c->page_size < (long long)c->max_blocks * c->block_size) return COBS_ERR_INVALID_ARG;
+  // the attention kernel indexes at most kMaxGroupsPerCta 16-token groups per CTA with at most kMaxSplits splits
+  if ((long long)max_items(c) * (c->block_size / 16) > (long long)kMaxGroupsPerCta * kMaxSplits) return COBS_ERR_UNSUPPORTED;
   return COBS_OK;
 }
 
+// Split-KV partials per (sequence, KV head): as many CTAs as fit in ONE wave (3 resident CTAs per SM,
+// so that no CTA waits for a second wave), never more than there are blocks to read, and few enough
+// groups per CTA for its index table.
 static int choose_splits(const cobs_config *c) {
   const int units = c->batch * c->n_kv_heads;
-  const int items = c->topk + (c->window + c->block_size - 1) / c->block_size + 1;
-  int s = (2 * 148 + units - 1) / units;
+  const int items = max_items(c);
+  int s = (3 * 148) / units;
+  const int need = (items * (c->block_size / 16) + kMaxGroupsPerCta - 1) / kMaxGroupsPerCta;
+  if (s < need) s = need;
   if (s > items) s = items;
   if (s > kMaxSplits) s = kMaxSplits;
   if (s < 1) s = 1;

@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(kScoreThreads, 4) score_mma_kernel(Params p, i
 #pragma unroll
       for (int m = 0; m < KSM / 2; ++m) {
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (gid < G) v = *reinterpret_cast<const uint4 *>(qg + gid * D + tig * (D / 4) + m * 8);
+        if (gid < G) v = *reinterpret_cast<const uint4 *>(qg + gid * D + (tig + 4 * m) * 8);
         bm[2 * m][0] = v.x; bm[2 * m][1] = v.y; bm[2 * m + 1][0] = v.z; bm[2 * m + 1][1] = v.w;
       }
       if (DT == COBS_SUMM_FP4_E2M1) {
@@ -167,11 +167,12 @@ __global__ void __launch_bounds__(kScoreThreads, 4) score_mma_kernel(Params p, i
     // ---- first-order term: the 16 block means against the raw bf16 query -------------------------
     float c[4] = {0.f, 0.f, 0.f, 0.f};
     {
-      const uint4 *ma = reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)p.mean + recA * D + tig * (D / 4));
-      const uint4 *mb = reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)p.mean + recB * D + tig * (D / 4));
+      // 16-byte chunk tig + 4 m of each row: the four lanes of a quad read 64 contiguous bytes
+      const uint4 *ma = reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)p.mean + recA * D) + tig;
+      const uint4 *mb = reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)p.mean + recB * D) + tig;
       uint4 va[KSM / 2], vb[KSM / 2];
 #pragma unroll
-      for (int m = 0; m < KSM / 2; ++m) { va[m] = ldg_stream(ma + m); vb[m] = ldg_stream(mb + m); }
+      for (int m = 0; m < KSM / 2; ++m) { va[m] = ldg_stream(ma + 4 * m); vb[m] = ldg_stream(mb + 4 * m); }
 #pragma unroll
       for (int m = 0; m < KSM / 2; ++m) {
         mma_bf16(c, va[m].x, vb[m].x, va[m].y, vb[m].y, bm[2 * m][0], bm[2 * m][1]);
@@ -183,14 +184,14 @@ __global__ void __launch_bounds__(kScoreThreads, 4) score_mma_kernel(Params p, i
 
     // ---- curvature term: sum_i (xi_i . q~)^2 ----------------------------------------------------------
     if (DT == COBS_SUMM_BF16) {
-      const __nv_bfloat16 *xa = (const __nv_bfloat16 *)p.xi + recA * r * D + tig * (D / 4);
-      const __nv_bfloat16 *xb = (const __nv_bfloat16 *)p.xi + recB * r * D + tig * (D / 4);
+      const __nv_bfloat16 *xa = (const __nv_bfloat16 *)p.xi + recA * r * D + tig * 8;
+      const __nv_bfloat16 *xb = (const __nv_bfloat16 *)p.xi + recB * r * D + tig * 8;
       for (int i = 0; i < r; ++i) {
         const uint4 *pa = reinterpret_cast<const uint4 *>(xa + (size_t)i * D);
         const uint4 *pb = reinterpret_cast<const uint4 *>(xb + (size_t)i * D);
         uint4 va[KSM / 2], vb[KSM / 2];
 #pragma unroll
-        for (int m = 0; m < KSM / 2; ++m) { va[m] = ldg_stream(pa + m); vb[m] = ldg_stream(pb + m); }
+        for (int m = 0; m < KSM / 2; ++m) { va[m] = ldg_stream(pa + 4 * m); vb[m] = ldg_stream(pb + 4 * m); }
         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int m = 0; m < KSM / 2; ++m) {

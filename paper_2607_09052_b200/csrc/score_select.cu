@@ -111,47 +111,74 @@ __global__ void __launch_bounds__(256) score_generic_kernel(Params p, int blocks
 // ------------------------------------------------------------------------------------------------
 // Group score + top-k, one CTA per (sequence, KV head).
 // ------------------------------------------------------------------------------------------------
-constexpr int kSelThreads = 256;
+constexpr int kSelThreads = 512;
+constexpr int kSelWarps = kSelThreads / 32;
 
-__device__ float block_reduce(float v, bool is_max, float *scratch) {
+// Exclusive prefix sum of one int per thread over the CTA (fixed order); *total gets the sum.
+__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_tot, int *total) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  v = is_max ? warp_max(v) : warp_sum(v);
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
   __syncthreads();
-  if (lane == 0) scratch[warp] = v;
+  if (lane == 31) warp_tot[warp] = inc;
   __syncthreads();
-  float r = scratch[0];
-  for (int w = 1; w < (int)(blockDim.x >> 5); ++w) r = is_max ? fmaxf(r, scratch[w]) : r + scratch[w];
-  return r;
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kSelWarps; ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) base += t;
+    tot += t;
+  }
+  *total = tot;
+  return base + inc - v;
 }
 
 __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p) {
   extern __shared__ float score[];                 // [NB]
-  __shared__ float scratch[kSelThreads / 32];
+  __shared__ float red_m[kSelWarps], red_s[kSelWarps];
   __shared__ float lse[8];
   __shared__ int hist[256];
-  __shared__ int counts[kSelThreads];
-  __shared__ int eq_base[kSelThreads];
+  __shared__ int warp_tot[kSelWarps];
   __shared__ uint32_t s_prefix;
   __shared__ int s_need;
 
-  const int u = blockIdx.x, b_idx = u / p.Hkv, tid = threadIdx.x;
+  const int u = blockIdx.x, b_idx = u / p.Hkv, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int T = p.seq_lens[b_idx];
   const int n_sum = min(T / p.L, p.NB);
   const int n_cand = min(window_start(T, p.window, p.L) / p.L, n_sum);
   const int G = p.G;
 
-  // log-sum-exp of each head's estimates over every summarised block
+  // log-sum-exp of each head's estimates over every summarised block: one pass of (max, sum) pairs
   for (int g = 0; g < G; ++g) {
     const float *e = p.e + ((size_t)u * G + g) * p.NB;
-    float mx = -INFINITY;
-    for (int b = tid; b < n_sum; b += kSelThreads) mx = fmaxf(mx, e[b]);
-    mx = block_reduce(mx, true, scratch);
-    float sm = 0.f;
-    for (int b = tid; b < n_sum; b += kSelThreads) sm += expf(e[b] - mx);
-    sm = block_reduce(sm, false, scratch);
-    if (tid == 0) lse[g] = mx + logf(sm);
+    float mx = -INFINITY, sm = 0.f;
+    for (int b = tid; b < n_sum; b += kSelThreads) {
+      const float x = e[b];
+      if (x > mx) { sm = sm * expf(mx - x) + 1.0f; mx = x; }
+      else sm += expf(x - mx);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, mx, o), os = __shfl_xor_sync(0xffffffffu, sm, o);
+      const float nm = fmaxf(mx, om);
+      sm = (nm == -INFINITY) ? 0.f : sm * expf(mx - nm) + os * expf(om - nm);
+      mx = nm;
+    }
+    if (lane == 0) { red_m[warp] = mx; red_s[warp] = sm; }
+    __syncthreads();
+    if (tid == 0) {
+      float M = -INFINITY;
+      for (int w = 0; w < kSelWarps; ++w) M = fmaxf(M, red_m[w]);
+      float S = 0.f;
+      for (int w = 0; w < kSelWarps; ++w) S += (red_m[w] == -INFINITY) ? 0.f : red_s[w] * expf(red_m[w] - M);
+      lse[g] = M + logf(S);
+    }
+    __syncthreads();
   }
-  __syncthreads();
   for (int b = tid; b < n_sum; b += kSelThreads) {
     float s = 0.f;
     for (int g = 0; g < G; ++g) s += expf(p.e[((size_t)u * G + g) * p.NB + b] - lse[g]);
@@ -178,18 +205,32 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p) {
     __syncthreads();
     const uint32_t prefix = s_prefix;
     for (int b = tid; b < n_cand; b += kSelThreads) {
-      uint32_t key = __float_as_uint(score[b]);
+      const uint32_t key = __float_as_uint(score[b]);
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
     }
     __syncthreads();
-    if (tid == 0) {
-      int need = s_need, cum = 0, bin = 255;
-      for (; bin > 0; --bin) {
-        if (cum + hist[bin] >= need) break;
-        cum += hist[bin];
+    if (warp == 0) {
+      // lane l owns bins 255 - 8 l ... 248 - 8 l (descending); find the bin where the running count reaches `need`
+      const int need = s_need;
+      int mine = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) mine += hist[255 - 8 * lane - j];
+      int inc = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
       }
-      s_need = need - cum;
-      s_prefix = prefix | ((uint32_t)bin << shift);
+      const int before = inc - mine;
+      if (before < need && inc >= need) {          // exactly one lane
+        int cum = before, bin = 255 - 8 * lane;
+        for (int j = 0; j < 8; ++j, --bin) {
+          if (cum + hist[bin] >= need) break;
+          cum += hist[bin];
+        }
+        s_need = need - cum;
+        s_prefix = prefix | ((uint32_t)bin << shift);
+      }
     }
     mask |= 255u << shift;
     __syncthreads();
@@ -202,31 +243,18 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Params p) {
   const int lo = min(tid * per, n_cand), hi = min(lo + per, n_cand);
   int n_eq = 0;
   for (int b = lo; b < hi; ++b) n_eq += (__float_as_uint(score[b]) == theta);
-  counts[tid] = n_eq;
-  __syncthreads();
-  if (tid == 0) {
-    int run = 0;
-    for (int i = 0; i < kSelThreads; ++i) { eq_base[i] = run; run += counts[i]; }
-  }
-  __syncthreads();
-  int eq_rank = eq_base[tid];
-  int n_keep = 0;
+  int total;
+  const int eq_base = block_exclusive_scan(n_eq, warp_tot, &total);
+  int eq_rank = eq_base, n_keep = 0;
   for (int b = lo; b < hi; ++b) {
-    uint32_t key = __float_as_uint(score[b]);
+    const uint32_t key = __float_as_uint(score[b]);
     if (key > theta) ++n_keep;
     else if (key == theta) { if (eq_rank < need_eq) ++n_keep; ++eq_rank; }
   }
-  counts[tid] = n_keep;
-  __syncthreads();
-  if (tid == 0) {
-    int run = 0;
-    for (int i = 0; i < kSelThreads; ++i) { int c = counts[i]; counts[i] = run; run += c; }
-  }
-  __syncthreads();
-  int pos = counts[tid];
-  eq_rank = eq_base[tid];
+  int pos = block_exclusive_scan(n_keep, warp_tot, &total);
+  eq_rank = eq_base;
   for (int b = lo; b < hi; ++b) {
-    uint32_t key = __float_as_uint(score[b]);
+    const uint32_t key = __float_as_uint(score[b]);
     bool keep = false;
     if (key > theta) keep = true;
     else if (key == theta) { keep = eq_rank < need_eq; ++eq_rank; }
