@@ -127,6 +127,10 @@ def run_ours(args):
     wl = synth.named_workloads()[args.workload]
     if args.batch:
         wl = wl.replace(batch=args.batch, name=f"{wl.name}[batch={args.batch}]")
+    if args.seq_len:
+        wl = wl.replace(seq_len=args.seq_len, name=f"{wl.name}[context={args.seq_len}]")
+    if args.contiguous_pages:
+        wl = wl.replace(shuffle_pages=False, name=f"{wl.name}[contiguous pages]")
     wl = wl.replace(seed=wl.seed + 1000 * rank)        # every rank draws its own sequences
     dev = torch.device("cuda", local_rank)
     inp = synth.generate(wl, dev)
@@ -382,6 +386,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a small case)")
+    ap.add_argument("--seq-len", type=int, default=0, help="override the workload's context (profiling on a small case)")
+    ap.add_argument("--contiguous-pages", action="store_true",
+                    help="diagnostic: identity page table instead of the workload's shuffled pages")
     ap.add_argument("--clock-warm-s", type=float, default=0.6,
                     help="keep warming up at least this long so that the clock sampler has samples")
     args = ap.parse_args()

@@ -12,7 +12,9 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_select(const Params &p, cudaStream_t stream);
-cudaError_t launch_attend(const Params &p, cudaStream_t stream);
+cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream);
+bool fused_score_supported(const Params &p);
+enum { PH_SCORE = 1, PH_ATTEND = 2 };
 cudaError_t launch_build(const Params &p, int block_begin, int block_end, cudaStream_t stream);
 cudaError_t launch_quantise(const float *xi, long long n_vectors, int Ds, int Ds_pad, int scale_dtype, void *codes,
                             void *scale, cudaStream_t stream);
@@ -25,7 +27,8 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 // every block starts on a 16-byte boundary.
 static int padded_sub_dim(int Ds, int /*r*/) { return (Ds + 31) / 32 * 32; }
 
-constexpr int kMaxGroupsPerCta = 1024;   // 16-token groups one attention CTA can index
+constexpr int kItemGroups = 256;         // 16-token groups one attention work item may hold
+constexpr int kGridWarps = 148 * 2 * 4;  // warps of the persistent kernel on a B200 (sizing heuristic only)
 
 static int max_items(const cobs_config *c) {
   return c->topk + (c->window + c->block_size - 1) / c->block_size + 1;
@@ -53,28 +56,29 @@ static int32_t validate_config(const cobs_config *c) {
   if (c->max_pages_per_seq < 1) return COBS_ERR_INVALID_ARG;
   // the page table must cover every token a sequence may hold: NB * L + L - 1 at most
   if ((long long)c->max_pages_per_seq * c->page_size < (long long)c->max_blocks * c->block_size) return COBS_ERR_INVALID_ARG;
-  // the attention kernel indexes at most kMaxGroupsPerCta 16-token groups per CTA with at most kMaxSplits splits
-  if ((long long)max_items(c) * (c->block_size / 16) > (long long)kMaxGroupsPerCta * kMaxSplits) return COBS_ERR_UNSUPPORTED;
+  // an attention slice holds at most kItemGroups 16-token groups and a unit at most kMaxSplits slices
+  if ((long long)max_items(c) * (c->block_size / 16) > (long long)kItemGroups * kMaxSplits) return COBS_ERR_UNSUPPORTED;
+  if ((long long)c->batch * c->n_kv_heads > kMaxUnits) return COBS_ERR_UNSUPPORTED;
   return COBS_OK;
 }
 
-// Split-KV partials per (sequence, KV head): as many CTAs as fit in ONE wave (3 resident CTAs per SM,
-// so that no CTA waits for a second wave), never more than there are blocks to read, and few enough
-// groups per CTA for its index table.
+// Attention slices per (sequence, KV head): one slice per warp of the persistent grid when the batch is
+// large enough for that, never more than there are 16-token groups to read, and enough that a slice
+// fits the kernel's per-warp group table.
 static int choose_splits(const cobs_config *c) {
   const int units = c->batch * c->n_kv_heads;
-  const int items = max_items(c);
-  int s = (3 * 148) / units;
-  const int need = (items * (c->block_size / 16) + kMaxGroupsPerCta - 1) / kMaxGroupsPerCta;
+  const int groups = max_items(c) * (c->block_size / 16);
+  int s = kGridWarps / units;
+  const int need = (groups + kItemGroups - 1) / kItemGroups;
   if (s < need) s = need;
-  if (s > items) s = items;
+  if (s > groups) s = groups;
   if (s > kMaxSplits) s = kMaxSplits;
   if (s < 1) s = 1;
   return s;
 }
 
 struct WorkspaceLayout {
-  size_t status, e, partial, sel_idx, sel_cnt, q_stage, out_stage, total;
+  size_t status, ctl, e, lse_part, partial, sel_idx, sel_cnt, qtilde, q_stage, out_stage, total;
 };
 
 static WorkspaceLayout layout_workspace(const cobs_config *c) {
@@ -82,10 +86,13 @@ static WorkspaceLayout layout_workspace(const cobs_config *c) {
   const size_t B = c->batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, G = Hq / Hkv, D = c->head_dim;
   size_t off = 0;
   w.status = off; off += kStatusBytes;
+  w.ctl = off; off = align_up(off + 3 * B * Hkv * sizeof(int), 256);     // inside the first kCtlBytes
   w.e = off; off = align_up(off + B * Hq * (size_t)c->max_blocks * sizeof(float), 256);
+  w.lse_part = off; off = align_up(off + B * Hq * (size_t)((c->max_blocks + 15) / 16) * 2 * sizeof(float), 256);
   w.partial = off; off = align_up(off + B * Hkv * (size_t)choose_splits(c) * G * (D + 2) * sizeof(float), 256);
   w.sel_idx = off; off = align_up(off + B * Hkv * (size_t)c->topk * sizeof(int32_t), 256);
   w.sel_cnt = off; off = align_up(off + B * Hkv * sizeof(int32_t), 256);
+  w.qtilde = off; off = align_up(off + (c->sub_dim ? B * Hq * (size_t)((c->sub_dim + 31) / 32 * 32) * sizeof(float) : 0), 256);
   w.q_stage = off; off = align_up(off + B * Hq * D * 2, 256);
   w.out_stage = off; off = align_up(off + B * Hq * D * sizeof(float), 256);
   w.total = off;
@@ -105,7 +112,13 @@ static void fill_params(Params &p, const cobs_config *c, void *workspace) {
     WorkspaceLayout w = layout_workspace(c);
     char *base = static_cast<char *>(workspace);
     p.status = reinterpret_cast<int32_t *>(base + w.status);
+    p.ctl_done = reinterpret_cast<int *>(base + w.status) + 1;
+    p.ctl_score = reinterpret_cast<int *>(base + w.ctl);
+    p.ctl_ready = p.ctl_score + (size_t)p.B * p.Hkv;
+    p.ctl_att = p.ctl_ready + (size_t)p.B * p.Hkv;
+    p.qtilde_out = reinterpret_cast<float *>(base + w.qtilde);
     p.e = reinterpret_cast<float *>(base + w.e);
+    p.lse_part = reinterpret_cast<float *>(base + w.lse_part);
     p.partial = reinterpret_cast<float *>(base + w.partial);
     p.sel_idx = reinterpret_cast<int32_t *>(base + w.sel_idx);
     p.sel_cnt = reinterpret_cast<int32_t *>(base + w.sel_cnt);
@@ -197,7 +210,8 @@ int32_t cobs_workspace_bytes(const cobs_config *cfg, size_t *bytes) {
 
 int32_t cobs_reset_status(void *workspace, size_t workspace_bytes, void *stream) {
   if (!workspace || workspace_bytes < (size_t)kStatusBytes) return COBS_ERR_INVALID_ARG;
-  return cuda_status(cudaMemsetAsync(workspace, 0, kStatusBytes, static_cast<cudaStream_t>(stream)));
+  const size_t n = workspace_bytes < (size_t)kCtlBytes ? workspace_bytes : (size_t)kCtlBytes;
+  return cuda_status(cudaMemsetAsync(workspace, 0, n, static_cast<cudaStream_t>(stream)));
 }
 
 int32_t cobs_read_status(void *workspace, size_t workspace_bytes, void *stream, int32_t *code_host) {
@@ -248,6 +262,10 @@ int32_t cobs_score_select(const cobs_config *cfg, const void *q, const cobs_summ
   p.seq_lens = seq_lens;
   p.sel_idx = sel_idx; p.sel_cnt = sel_cnt; p.scores = scores_or_null;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (fused_score_supported(p)) {
+    if (p.u_q) p.qtilde = p.qtilde_out;
+    return cuda_status(launch_fused(p, PH_SCORE, s));
+  }
   cudaError_t e = launch_score(p, s);
   if (e != cudaSuccess) return COBS_ERR_CUDA;
   return cuda_status(launch_select(p, s));
@@ -266,7 +284,7 @@ int32_t cobs_sparse_decode(const cobs_config *cfg, const void *q, const cobs_kv 
   p.q = static_cast<const __nv_bfloat16 *>(q);
   p.sel_idx = const_cast<int32_t *>(sel_idx); p.sel_cnt = const_cast<int32_t *>(sel_cnt);
   p.out = out; p.lse = lse_or_null;
-  return cuda_status(launch_attend(p, static_cast<cudaStream_t>(stream)));
+  return cuda_status(launch_fused(p, PH_ATTEND, static_cast<cudaStream_t>(stream)));
 }
 
 int32_t cobs_decode_step(const cobs_config *cfg, const void *q, const cobs_kv *kv, const cobs_summaries *summ,
@@ -285,10 +303,16 @@ int32_t cobs_decode_step(const cobs_config *cfg, const void *q, const cobs_kv *k
   if (sel_idx_or_null) { p.sel_idx = sel_idx_or_null; p.sel_cnt = sel_cnt_or_null; }
   p.out = out; p.lse = lse_or_null;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (fused_score_supported(p)) {
+    if (p.u_q) p.qtilde = p.qtilde_out;
+    return cuda_status(launch_fused(p, PH_SCORE | PH_ATTEND, s));
+  }
+  // summaries the persistent kernel's scoring phase does not cover (fp32, odd subspace widths):
+  // generic scoring and selection kernels first, then the persistent kernel for the attention
   cudaError_t e = launch_score(p, s);
   if (e != cudaSuccess) return COBS_ERR_CUDA;
   if ((e = launch_select(p, s)) != cudaSuccess) return COBS_ERR_CUDA;
-  return cuda_status(launch_attend(p, s));
+  return cuda_status(launch_fused(p, PH_ATTEND, s));
 }
 
 int32_t cobs_decode_step_host(const cobs_config *cfg, const void *q_host, const cobs_kv *kv,

@@ -11,7 +11,9 @@
 namespace cobs {
 
 constexpr int kStatusBytes = 256;          // status word lives in the first 256 bytes of the workspace
-constexpr int kMaxSplits = 32;             // upper bound on split-KV partials per (sequence, KV head)
+constexpr int kMaxSplits = 64;             // upper bound on split-KV partials per (sequence, KV head)
+constexpr int kMaxUnits = 65536;           // (sequence, KV head) units a workspace has counters for
+constexpr int kCtlBytes = kStatusBytes + 3 * kMaxUnits * 4;   // status word + counters, zeroed by cobs_reset_status
 
 // Everything a kernel needs, passed by value.
 struct Params {
@@ -30,7 +32,14 @@ struct Params {
   const float *u_q;
   // workspace pieces
   int32_t *status;
+  int *ctl_done;              // CTAs of the persistent kernel that have finished
+  int *ctl_score;             // [B * Hkv] scored chunks per unit
+  int *ctl_ready;             // [B * Hkv] 1 once the unit's selection is written
+  int *ctl_att;               // [B * Hkv] attention slices finished per unit
+  const float *qtilde;        // [B][Hq][Ds_pad] prepared subspace query, or NULL
+  float *qtilde_out;
   float *e;                   // [B][Hkv][G][NB]
+  float *lse_part;            // [B][Hkv][G][ceil(NB / 16)][2] per-chunk (max, sum-exp) of e
   float *partial;             // [B][Hkv][n_splits][G][D + 2]
   int32_t *sel_idx;           // [B][Hkv][topk]
   int32_t *sel_cnt;           // [B][Hkv]

@@ -1,0 +1,997 @@
+// The decode step as ONE persistent kernel: block scoring, top-k selection, block-sparse attention
+// and the split-KV merge (steps (b), (c), (d)).
+//
+// Why one kernel.  A step moves a few hundred MiB; at HBM speed that is tens of microseconds, so
+// every kernel boundary (launch, ramp-up, tail, the idle time while a single CTA per unit selects)
+// costs a visible fraction of the step.  Here the grid is sized to be fully resident (2 CTAs of 4
+// warps per SM) and every WARP runs the same program on its own share of the work:
+//
+//   phase S  score 16-block chunks of summaries (chunks dealt round-robin to all warps of the grid,
+//            so the grid sweeps the summary arrays front to back and units finish in order);
+//            the warp that finishes the last chunk of a (sequence, KV head) unit selects its top-k;
+//   phase A  attend over (unit, split) items, dealt round-robin in unit order; a warp whose slice
+//            holds selected blocks waits (bounded) for that unit's selection, slices that hold only
+//            window blocks never wait; the warp that finishes the last slice of a unit merges the
+//            partials and writes the output.
+//
+// Data movement.  Every stream a warp consumes goes global -> shared with cp.async into a ring that
+// belongs to that warp alone (no CTA barrier anywhere in the loops) and ALL streams of a phase have
+// the same prefetch depth: a shallower stream would set the pace while the deeper ones only add
+// queueing delay.  Scoring: thread-private 16-byte slots (a lane copies exactly the fragments it will
+// feed to the tensor core), depth 1.  Attention: K and V of a 16-token group share a stage
+// (XOR-swizzled 16-byte chunks, read back with ldmatrix / ldmatrix.trans), depth 2.
+//
+// Arithmetic.  mma.sync m16n8k16 with fp32 accumulation throughout:
+//   scoring   rows = 16 block means, or factor i of 16 blocks; columns = the G query heads.  A thread
+//             owns two blocks (rows gid, gid + 8), so all results of a block land in one thread.
+//             bf16 operands multiply the raw bf16 query (exact products); FP4 codes become f16 by
+//             the hardware conversion and multiply the query scaled by a per-head power of two
+//             (exact in f16), or an f16 high + low split of the fp32 subspace query.
+//   attention S^T = q K^T with the heads as rows (zero padded to 16) and 8 tokens as columns; the S
+//             accumulators are the A fragments of P V as they sit in registers; P = bf16 high + low.
+//
+// Cross-warp hand-offs go through global counters in the workspace (release: write, __threadfence,
+// atomicAdd; acquire: volatile read, __threadfence, .cg loads).  Every wait is bounded; on expiry the
+// kernel records COBS_ERR_TIMEOUT, skips the dependent work and returns.  The last CTA to finish puts
+// the counters back to zero, so a workspace needs zeroing only once (cobs_reset_status).
+#include "common.cuh"
+
+namespace cobs {
+
+constexpr int kFWarps = 4;
+constexpr int kFThreads = kFWarps * 32;
+constexpr int kSlots = 24;                                   // 16-byte slots per lane per scoring stage
+constexpr int kScaleBytes = 16 * COBS_MAX_RANK * 4;          // scales of a chunk (16 blocks x r, fp32)
+constexpr int kScoreStageBytes = kSlots * 512 + kScaleBytes; // 13312
+constexpr int kAttStages = 3;
+constexpr int kAttStageBytes = 2 * 16 * 128 * 2;             // K + V of one 16-token group, D = 128
+constexpr int kHistBytes = 1024;
+constexpr int kTableEntries = 256;                           // 16-token groups per attention item
+constexpr int kRingBytes = (2 * kScoreStageBytes > kAttStages * kAttStageBytes + kTableEntries * 8)
+                               ? 2 * kScoreStageBytes : kAttStages * kAttStageBytes + kTableEntries * 8;
+constexpr int kWarpSmemBytes = kRingBytes + kHistBytes;      // 27648
+constexpr int kFusedSmemBytes = kFWarps * kWarpSmemBytes;    // 110592
+constexpr int kMaxSelectBlocks = 16384;                      // scores + chunk weights of a unit fit the CTA's shared memory
+constexpr long long kSpinLimit = 4000000;                    // x ~100 ns: bounded wait on another warp
+
+enum { PH_SCORE = 1, PH_ATTEND = 2 };
+
+// ---------------------------------------------------------------------------------------------------
+// small PTX helpers
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cpa16(uint32_t dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src));
+}
+__device__ __forceinline__ void cpa16z(uint32_t dst, const void *src, int bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(bytes));
+}
+__device__ __forceinline__ void cpa4(uint32_t dst, const void *src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(dst), "l"(src));
+}
+__device__ __forceinline__ void cpa_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cpa_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void mma16816_bf16(float &c0, float &c1, float &c2, float &c3, uint32_t a0, uint32_t a1,
+                                              uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma16816_f16(float &c0, float &c1, float &c2, float &c3, uint32_t a0, uint32_t a1,
+                                             uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// Eight E2M1 codes -> four f16x2 (code 2 i in the low half of h[i], code 2 i + 1 in the high half).
+__device__ __forceinline__ void e2m1x8_to_f16(uint32_t w, uint32_t (&h)[4]) {
+  asm("{\n .reg .b8 b0, b1, b2, b3;\n mov.b32 {b0, b1, b2, b3}, %4;\n cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+      " cvt.rn.f16x2.e2m1x2 %1, b1;\n cvt.rn.f16x2.e2m1x2 %2, b2;\n cvt.rn.f16x2.e2m1x2 %3, b3;\n}\n"
+      : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]) : "r"(w));
+}
+__device__ __forceinline__ uint32_t f16x2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t *>(&h);
+}
+__device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ int ld_volatile(const int *p) { return *reinterpret_cast<const volatile int *>(p); }
+
+// Wait until *flag != 0 (set by another warp of the grid).  Bounded; false on expiry.
+__device__ __forceinline__ bool wait_flag(const int *flag) {
+  for (long long it = 0; it < kSpinLimit; ++it) {
+    if (ld_volatile(flag) != 0) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Selection phase.  Unit u is selected by CTA u mod gridDim.x (all four warps together) once all its
+// chunks are scored.  Scoring left, per block, t = exp(e - chunk max) and, per chunk, (max, sum of t):
+//   lse_g   = log-sum-exp over the chunks of head g
+//   score_b = sum_g t[g][b] * exp(chunk max[g] - lse_g)          (= sum_g exp(e[g][b] - lse_g))
+// then the k largest scores among the candidate blocks, lower index on ties, ascending output.
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int cta_exclusive_scan(int v, int *warp_tot, int *total) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kFWarps; ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) base += t;
+    tot += t;
+  }
+  *total = tot;
+  return base + inc - v;
+}
+
+__device__ void select_phase(const Params &p, unsigned char *cta_smem) {
+  __shared__ float s_w[8][kFWarps];          // per head: per-warp (max, sum) while reducing, then the lse
+  __shared__ float s_w2[8][kFWarps];
+  __shared__ float s_lse[8];
+  __shared__ int s_hist[256];
+  __shared__ int s_tot[kFWarps];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_need, s_ok;
+  float *sc = reinterpret_cast<float *>(cta_smem);             // [NB] scores; the rings are idle in this phase
+  float *cw = sc + p.NB;                                       // [G][chunks] exp(chunk max - lse)
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int units = p.B * p.Hkv, G = p.G, NB = p.NB, cpu = (NB + 15) / 16;
+
+  for (int u = blockIdx.x; u < units; u += gridDim.x) {
+    const int T = p.seq_lens[u / p.Hkv];
+    const int n_sum = min(T / p.L, NB);
+    const int n_cand = min(window_start(T, p.window, p.L) / p.L, n_sum);
+    const int n_chunks = (n_sum + 15) / 16;
+    if (tid == 0) {
+      int ok = 0;
+      for (long long it = 0; it < kSpinLimit; ++it) {
+        if (ld_volatile(p.ctl_score + u) >= max(n_chunks, 1)) { ok = 1; break; }
+        __nanosleep(100);
+      }
+      if (!ok) report(p.status, COBS_ERR_TIMEOUT);
+      s_ok = ok;
+    }
+    __syncthreads();
+    if (!s_ok) { __syncthreads(); continue; }                  // never scored: leave the unit unselected
+    __threadfence();
+
+    // ---- lse per head from the chunk pairs ------------------------------------------------------------
+    const float2 *pp = reinterpret_cast<const float2 *>(p.lse_part) + (size_t)u * G * cpu;
+    for (int g = 0; g < G; ++g) {
+      float m = -INFINITY, s = 0.f;
+      for (int c = tid; c < n_chunks; c += kFThreads) {
+        const float2 v = __ldcg(pp + (size_t)g * cpu + c);
+        const float nm = fmaxf(m, v.x);
+        s = s * expf(m - nm) + v.y * expf(v.x - nm);
+        m = nm;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+        const float nm = fmaxf(m, om);
+        s = (nm == -INFINITY) ? 0.f : s * expf(m - nm) + os * expf(om - nm);
+        m = nm;
+      }
+      if (lane == 0) { s_w[g][warp] = m; s_w2[g][warp] = s; }
+    }
+    __syncthreads();
+    if (tid < G) {
+      float M = -INFINITY;
+      for (int w = 0; w < kFWarps; ++w) M = fmaxf(M, s_w[tid][w]);
+      float S = 0.f;
+      for (int w = 0; w < kFWarps; ++w) S += (s_w[tid][w] == -INFINITY) ? 0.f : s_w2[tid][w] * expf(s_w[tid][w] - M);
+      s_lse[tid] = M + logf(S);
+    }
+    __syncthreads();
+    for (int i = tid; i < G * n_chunks; i += kFThreads) {
+      const int g = i / n_chunks, c = i - g * n_chunks;
+      cw[g * cpu + c] = expf(__ldcg(pp + (size_t)g * cpu + c).x - s_lse[g]);
+    }
+    __syncthreads();
+    // ---- scores -------------------------------------------------------------------------------------------
+    const float *tu = p.e + (size_t)u * G * NB;
+    for (int b0 = 0; b0 < n_sum; b0 += 4 * kFThreads) {
+      float x[8][4];
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int b = b0 + tid + kFThreads * j;
+          x[g][j] = (g < G && b < n_sum) ? __ldcg(tu + (size_t)g * NB + b) : 0.f;
+        }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int b = b0 + tid + kFThreads * j;
+        if (b < n_sum) {
+          float sv = 0.f;
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            if (g < G) sv = fmaf(x[g][j], cw[g * cpu + (b >> 4)], sv);
+          sc[b] = sv;
+          if (p.scores) p.scores[(size_t)u * NB + b] = sv;
+        }
+      }
+    }
+    __syncthreads();
+
+    // ---- top-k -----------------------------------------------------------------------------------------------
+    int32_t *out = p.sel_idx + (size_t)u * p.topk;
+    const int k = min(p.topk, n_cand);
+    if (tid == 0) p.sel_cnt[u] = k;
+    for (int i = k + tid; i < p.topk; i += kFThreads) out[i] = -1;
+    if (k == n_cand) {
+      for (int i = tid; i < k; i += kFThreads) out[i] = i;
+    } else if (k > 0) {
+      // radix select of the k-th largest key (scores are >= 0: their bit patterns order like integers)
+      if (tid == 0) { s_prefix = 0u; s_need = k; }
+      uint32_t mask = 0u;
+      for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = tid; i < 256; i += kFThreads) s_hist[i] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        for (int b = tid; b < n_cand; b += kFThreads) {
+          const uint32_t key = __float_as_uint(sc[b]);
+          if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        if (warp == 0) {
+          // lane l owns bins 255 - 8 l ... 248 - 8 l; find the bin where the count from the top reaches `need`
+          const int need = s_need;
+          int mine = 0;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) mine += s_hist[255 - 8 * lane - j];
+          int inc = mine;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+          }
+          const int before = inc - mine;
+          if (before < need && inc >= need) {              // exactly one lane
+            int cum = before, bin = 255 - 8 * lane;
+            for (int j = 0; j < 8; ++j, --bin) {
+              if (cum + s_hist[bin] >= need) break;
+              cum += s_hist[bin];
+            }
+            s_need = need - cum;
+            s_prefix = prefix | ((uint32_t)bin << shift);
+          }
+        }
+        mask |= 255u << shift;
+        __syncthreads();
+      }
+      const uint32_t theta = s_prefix;   // key of the k-th largest score
+      const int need_eq = s_need;        // blocks with exactly that key to keep (lowest indices first)
+      // ordered compaction: each thread owns a contiguous index range
+      const int per = (n_cand + kFThreads - 1) / kFThreads;
+      const int lo = min(tid * per, n_cand), hi = min(lo + per, n_cand);
+      int n_eq = 0;
+      for (int b = lo; b < hi; ++b) n_eq += (__float_as_uint(sc[b]) == theta);
+      int total;
+      const int eq_base = cta_exclusive_scan(n_eq, s_tot, &total);
+      int eq_rank = eq_base, n_keep = 0;
+      for (int b = lo; b < hi; ++b) {
+        const uint32_t key = __float_as_uint(sc[b]);
+        if (key > theta) ++n_keep;
+        else if (key == theta) { if (eq_rank < need_eq) ++n_keep; ++eq_rank; }
+      }
+      int pos = cta_exclusive_scan(n_keep, s_tot, &total);
+      eq_rank = eq_base;
+      for (int b = lo; b < hi; ++b) {
+        const uint32_t key = __float_as_uint(sc[b]);
+        bool keep = false;
+        if (key > theta) keep = true;
+        else if (key == theta) { keep = eq_rank < need_eq; ++eq_rank; }
+        if (keep && pos < k) out[pos++] = b;
+      }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) atomicExch(p.ctl_ready + u, 1);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// phase S: scoring (+ selection by the warp that completes a unit)
+// DT: COBS_SUMM_BF16 | COBS_SUMM_FP4_E2M1.  WPT: 32-bit words of codes per thread per FP4 row
+// (Ds_pad / 32).  NT: f16 terms of the query (1: full space, 2: fp32 subspace query).
+// ---------------------------------------------------------------------------------------------------
+template <int DT, int D, int WPT, int NT>
+__device__ void score_phase(const Params &p, unsigned char *wsm, int wg, int n_wg, int lane) {
+  constexpr bool FP4 = (DT == COBS_SUMM_FP4_E2M1);
+  constexpr int MCH = D / 32;                 // 16-byte chunks of a bf16 row per thread
+  constexpr int MEAN_SLOTS = 2 * MCH;         // two blocks
+  constexpr int ROW_SLOTS = FP4 ? 2 : 2 * MCH;
+  constexpr int ROWS0 = (kSlots - MEAN_SLOTS) / ROW_SLOTS;   // factor rows that fit beside the means
+  constexpr int ROWSN = kSlots / ROW_SLOTS;                  // factor rows of a later batch
+  constexpr int KSM = D / 16;                 // k-steps of a bf16 row
+  constexpr int KSQ = FP4 ? WPT * 2 : 1;      // k-steps of an FP4 row
+  const int gid = lane >> 2, tig = lane & 3;
+  const int G = p.G, r = p.r, NB = p.NB, L = p.L;
+  const int units = p.B * p.Hkv;
+  const int cpu = (NB + 15) / 16;             // chunks per unit
+  const long long total = (long long)units * cpu;
+  const int n_batches = (r <= ROWS0) ? 1 : 1 + (r - ROWS0 + ROWSN - 1) / ROWSN;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(wsm);
+  const float inv_sqrt_d = 1.0f / sqrtf((float)D);
+  const float ln_l = logf((float)L);
+  const int row_bytes = FP4 ? p.Ds_pad / 2 : D * 2;
+  const int scale_sz = (p.scale_dtype == COBS_SCALE_FP16) ? 2 : 4;
+
+  // position in this warp's batch sequence: chunk c (global index), batch b
+  auto chunk_valid = [&](long long c, int &u, int &n_sum) -> bool {
+    if (c >= total) return false;
+    u = (int)(c / cpu);
+    n_sum = min(p.seq_lens[u / p.Hkv] / L, NB);
+    const int ck = (int)(c - (long long)u * cpu);
+    // chunk 0 of a unit without summarised blocks is still visited: its warp publishes the empty selection
+    return ck * 16 < n_sum || ck == 0;
+  };
+  // this warp's contiguous range of chunks (mostly one unit: its query fragments are built once)
+  const long long per_warp = (total + n_wg - 1) / n_wg;
+  const long long c_begin = min((long long)wg * per_warp, total), c_end = min(c_begin + per_warp, total);
+  auto next_chunk = [&](long long c) -> long long {
+    int u, n;
+    while (c < c_end && !chunk_valid(c, u, n)) c = (long long)(u + 1) * cpu;   // rest of the unit has no summaries
+    return c < c_end ? c : total;
+  };
+
+  // ---- issue the copies of (chunk c, batch b) into stage st -----------------------------------------
+  auto issue = [&](long long c, int b, int st) {
+    if (c < total) {
+      const int u = (int)(c / cpu), ck = (int)(c - (long long)u * cpu);
+      const int n_sum = min(p.seq_lens[u / p.Hkv] / L, NB);
+      if (ck * 16 < n_sum) {
+        const int bA = min(ck * 16 + 2 * gid, NB - 1), bB = min(ck * 16 + 2 * gid + 1, NB - 1);
+        const size_t rec[2] = {(size_t)u * NB + bA, (size_t)u * NB + bB};
+        const uint32_t base = ring + st * kScoreStageBytes + lane * 16;
+        int slot = 0;
+        if (b == 0) {
+#pragma unroll
+          for (int a = 0; a < 2; ++a) {
+            const char *src = (const char *)p.mean + rec[a] * (size_t)(D * 2) + tig * 16;
+#pragma unroll
+            for (int m = 0; m < MCH; ++m) cpa16(base + (a * MCH + m) * 512, src + m * 64);
+          }
+          slot = MEAN_SLOTS;
+        }
+        if (FP4) {        // scales of the two blocks of this quad (every batch: a batch may sit in either stage)
+          const uint32_t sbase = ring + st * kScoreStageBytes + kSlots * 512;
+          const int per_blk = r * scale_sz;                    // bytes per block, a multiple of 4
+#pragma unroll
+          for (int a = 0; a < 2; ++a) {
+            const char *src = (const char *)p.scale + rec[a] * (size_t)per_blk;
+            for (int w = tig * 4; w < per_blk; w += 16) cpa4(sbase + (2 * gid + a) * 64 + w, src + w);
+          }
+        }
+        const int row0 = (b == 0) ? 0 : ROWS0 + (b - 1) * ROWSN;
+        const int rows = min(r - row0, (b == 0) ? ROWS0 : ROWSN);
+        for (int i = 0; i < rows; ++i) {
+#pragma unroll
+          for (int a = 0; a < 2; ++a) {
+            const char *src = (const char *)p.xi + (rec[a] * r + row0 + i) * (size_t)row_bytes;
+            if (FP4) {
+              const uint32_t dst = base + (slot + i * 2 + a) * 512;
+              if (WPT == 4) cpa16(dst, src + tig * 16);
+              else {
+#pragma unroll
+                for (int w = 0; w < WPT; ++w) cpa4(dst + w * 4, src + (tig * WPT + w) * 4);
+              }
+            } else {
+#pragma unroll
+              for (int m = 0; m < MCH; ++m) cpa16(base + (slot + (i * 2 + a) * MCH + m) * 512, src + tig * 16 + m * 64);
+            }
+          }
+        }
+      }
+    }
+    cpa_commit();
+  };
+
+  long long cur = next_chunk(c_begin);
+  int cur_b = 0, st = 0;
+  int pend_u = -1, pend_n = 0;              // chunks finished but not yet counted (counted once per unit run)
+  issue(cur, 0, 0);
+  // per-chunk state
+  uint32_t bm[KSM][2];
+  uint32_t bq[FP4 ? NT : 1][KSQ][2];
+  float m0 = 0.f, m1 = 0.f;
+  float fA0 = 0.f, fA1 = 0.f, fB0 = 0.f, fB1 = 0.f, sA0 = 0.f, sA1 = 0.f, sB0 = 0.f, sB1 = 0.f;
+  int cur_u = -1;
+
+  while (cur < total) {
+    // ---- prefetch the next batch of this warp --------------------------------------------------------
+    long long nxt = cur;
+    int nxt_b = cur_b + 1;
+    if (nxt_b >= n_batches) { nxt_b = 0; nxt = next_chunk(cur + 1); }
+    issue(nxt, nxt_b, st ^ 1);
+    cpa_wait<1>();
+    __syncwarp();
+
+    const int u = (int)(cur / cpu), ck = (int)(cur - (long long)u * cpu);
+    const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
+    const int n_sum = min(p.seq_lens[b_idx] / L, NB);
+    const uint32_t base = ring + st * kScoreStageBytes + lane * 16;
+    if (ck * 16 < n_sum) {
+      if (cur_b == 0) {
+        if (u != cur_u) {
+          cur_u = u;
+          // ---- query fragments of this unit ------------------------------------------------------------
+          const __nv_bfloat16 *qg = p.q + ((size_t)b_idx * p.Hq + h * G) * D;
+#pragma unroll
+          for (int m = 0; m < KSM / 2; ++m) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (gid < G) v = *reinterpret_cast<const uint4 *>(qg + gid * D + (tig + 4 * m) * 8);
+            bm[2 * m][0] = v.x; bm[2 * m][1] = v.y; bm[2 * m + 1][0] = v.z; bm[2 * m + 1][1] = v.w;
+          }
+          if (FP4) {
+            // this thread's WPT * 8 query elements of head gid: the raw bf16 query (full space; the
+            // 1/sqrt(D) factor is applied to the tile result) or the prepared fp32 q~ (subspace)
+            float e[WPT][8];
+            float mx = 0.f;
+#pragma unroll
+            for (int j = 0; j < WPT; ++j) {
+#pragma unroll
+              for (int n = 0; n < 8; ++n) {
+                float v = 0.f;
+                const int idx = tig * (WPT * 8) + j * 8 + n;
+                if (gid < G) {
+                  if (p.qtilde) v = p.qtilde[((size_t)b_idx * p.Hq + h * G + gid) * p.Ds_pad + idx];
+                  else v = __bfloat162float(qg[gid * D + idx]);
+                }
+                e[j][n] = v;
+                mx = fmaxf(mx, fabsf(v));
+              }
+            }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            int ex = 0;
+            if (mx > 0.f) frexpf(mx, &ex);
+            const float inv_s = ldexpf(1.0f, 1 - ex);       // power of two bringing max |q| into [1, 2)
+            const float mult = ldexpf(1.0f, ex - 1) * (p.qtilde ? 1.0f : inv_sqrt_d);
+#pragma unroll
+            for (int j = 0; j < WPT; ++j) {
+#pragma unroll
+              for (int t = 0; t < NT; ++t) {
+                float hi[8];
+#pragma unroll
+                for (int n = 0; n < 8; ++n) {
+                  hi[n] = __half2float(__float2half_rn(e[j][n] * (t == 0 ? inv_s : 1.0f)));
+                  e[j][n] = e[j][n] * (t == 0 ? inv_s : 1.0f) - hi[n];
+                }
+                bq[t][2 * j][0] = f16x2(hi[0], hi[1]); bq[t][2 * j][1] = f16x2(hi[2], hi[3]);
+                bq[t][2 * j + 1][0] = f16x2(hi[4], hi[5]); bq[t][2 * j + 1][1] = f16x2(hi[6], hi[7]);
+              }
+            }
+            // head 2 tig, 2 tig + 1 of the result columns belong to the lanes gid = 2 tig, 2 tig + 1 of any quad
+            m0 = __shfl_sync(0xffffffffu, mult, (2 * tig) * 4);
+            m1 = __shfl_sync(0xffffffffu, mult, (2 * tig + 1) * 4);
+          }
+        }
+        // ---- first-order term: block means against the raw bf16 query ------------------------------------
+        float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+#pragma unroll
+        for (int m = 0; m < MCH; ++m) {
+          const uint4 va = lds128(base + m * 512), vb = lds128(base + (MCH + m) * 512);
+          mma16816_bf16(c0, c1, c2, c3, va.x, vb.x, va.y, vb.y, bm[2 * m][0], bm[2 * m][1]);
+          mma16816_bf16(c0, c1, c2, c3, va.z, vb.z, va.w, vb.w, bm[2 * m + 1][0], bm[2 * m + 1][1]);
+        }
+        fA0 = c0 * inv_sqrt_d; fA1 = c1 * inv_sqrt_d; fB0 = c2 * inv_sqrt_d; fB1 = c3 * inv_sqrt_d;
+        sA0 = sA1 = sB0 = sB1 = 0.f;
+      }
+      // ---- curvature term: rows of this batch ----------------------------------------------------------
+      const int slot0 = (cur_b == 0) ? MEAN_SLOTS : 0;
+      const int row0 = (cur_b == 0) ? 0 : ROWS0 + (cur_b - 1) * ROWSN;
+      const int rows = min(r - row0, (cur_b == 0) ? ROWS0 : ROWSN);
+      const uint32_t sbase = ring + st * kScoreStageBytes + kSlots * 512 + (2 * gid) * 64;
+#pragma unroll
+      for (int i = 0; i < ROWSN; ++i) {
+        if (i < rows) {
+          float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+          if (FP4) {
+            uint32_t wa[4], wb[4];
+            if (WPT == 4) {
+              const uint4 a = lds128(base + (slot0 + i * 2) * 512), bb = lds128(base + (slot0 + i * 2 + 1) * 512);
+              wa[0] = a.x; wa[1] = a.y; wa[2] = a.z; wa[3] = a.w;
+              wb[0] = bb.x; wb[1] = bb.y; wb[2] = bb.z; wb[3] = bb.w;
+            } else {
+              const uint4 a = lds128(base + (slot0 + i * 2) * 512), bb = lds128(base + (slot0 + i * 2 + 1) * 512);
+              wa[0] = a.x; wa[1] = a.y; wa[2] = a.z; wa[3] = 0u;
+              wb[0] = bb.x; wb[1] = bb.y; wb[2] = bb.z; wb[3] = 0u;
+            }
+#pragma unroll
+            for (int j = 0; j < WPT; ++j) {
+              uint32_t ha[4], hb[4];
+              e2m1x8_to_f16(wa[j], ha);
+              e2m1x8_to_f16(wb[j], hb);
+#pragma unroll
+              for (int t = 0; t < NT; ++t) {
+                mma16816_f16(d0, d1, d2, d3, ha[0], hb[0], ha[1], hb[1], bq[t][2 * j][0], bq[t][2 * j][1]);
+                mma16816_f16(d0, d1, d2, d3, ha[2], hb[2], ha[3], hb[3], bq[t][2 * j + 1][0], bq[t][2 * j + 1][1]);
+              }
+            }
+            float sa, sb;
+            if (scale_sz == 4) {
+              sa = lds_f32(sbase + (row0 + i) * 4);
+              sb = lds_f32(sbase + 64 + (row0 + i) * 4);
+            } else {
+              const unsigned char *sp = wsm + st * kScoreStageBytes + kSlots * 512 + (2 * gid) * 64;
+              sa = __half2float(reinterpret_cast<const __half *>(sp)[row0 + i]);
+              sb = __half2float(reinterpret_cast<const __half *>(sp + 64)[row0 + i]);
+            }
+            d0 *= sa * m0; d1 *= sa * m1; d2 *= sb * m0; d3 *= sb * m1;
+          } else {
+#pragma unroll
+            for (int m = 0; m < MCH; ++m) {
+              const uint4 va = lds128(base + (slot0 + (i * 2) * MCH + m) * 512);
+              const uint4 vb = lds128(base + (slot0 + (i * 2 + 1) * MCH + m) * 512);
+              mma16816_bf16(d0, d1, d2, d3, va.x, vb.x, va.y, vb.y, bm[2 * m][0], bm[2 * m][1]);
+              mma16816_bf16(d0, d1, d2, d3, va.z, vb.z, va.w, vb.w, bm[2 * m + 1][0], bm[2 * m + 1][1]);
+            }
+            d0 *= inv_sqrt_d; d1 *= inv_sqrt_d; d2 *= inv_sqrt_d; d3 *= inv_sqrt_d;
+          }
+          sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
+        }
+      }
+    }
+
+    // ---- end of a chunk: publish t = exp(e - chunk max) per block and the chunk's (max, sum of t) per head ----
+    if (cur_b == n_batches - 1) {
+      if (pend_u != u && pend_n > 0) {       // moving on to another unit: count the finished one's chunks
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
+        pend_n = 0;
+      }
+      pend_u = u;
+      if (ck * 16 < n_sum) {
+        const int bA = ck * 16 + 2 * gid, bB = bA + 1, g0 = 2 * tig, g1 = g0 + 1;
+        const float eA0 = (bA < n_sum) ? ln_l + fA0 + 0.5f * sA0 : -INFINITY;
+        const float eB0 = (bB < n_sum) ? ln_l + fB0 + 0.5f * sB0 : -INFINITY;
+        const float eA1 = (bA < n_sum) ? ln_l + fA1 + 0.5f * sA1 : -INFINITY;
+        const float eB1 = (bB < n_sum) ? ln_l + fB1 + 0.5f * sB1 : -INFINITY;
+        // max over the chunk's 16 blocks (over gid), per head
+        float mx0 = fmaxf(eA0, eB0), mx1 = fmaxf(eA1, eB1);
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+        }
+        const float tA0 = expf(eA0 - mx0), tB0 = expf(eB0 - mx0), tA1 = expf(eA1 - mx1), tB1 = expf(eB1 - mx1);
+        float *e0 = p.e + ((size_t)u * G + g0) * NB, *e1 = p.e + ((size_t)u * G + g1) * NB;
+        if (g0 < G) {
+          if (bA < n_sum) __stcg(e0 + bA, tA0);
+          if (bB < n_sum) __stcg(e0 + bB, tB0);
+        }
+        if (g1 < G) {
+          if (bA < n_sum) __stcg(e1 + bA, tA1);
+          if (bB < n_sum) __stcg(e1 + bB, tB1);
+        }
+        float sm0 = tA0 + tB0, sm1 = tA1 + tB1;
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          sm0 += __shfl_xor_sync(0xffffffffu, sm0, o);
+          sm1 += __shfl_xor_sync(0xffffffffu, sm1, o);
+        }
+        if (gid == 0) {
+          if (g0 < G) __stcg(reinterpret_cast<float2 *>(p.lse_part) + ((size_t)u * G + g0) * cpu + ck, make_float2(mx0, sm0));
+          if (g1 < G) __stcg(reinterpret_cast<float2 *>(p.lse_part) + ((size_t)u * G + g1) * cpu + ck, make_float2(mx1, sm1));
+        }
+      }
+      ++pend_n;
+    }
+    __syncwarp();
+    cur = nxt; cur_b = nxt_b; st ^= 1;
+  }
+  cpa_wait<0>();
+  if (pend_n > 0) {
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// phase A: attention over (unit, split) items + merge
+// ---------------------------------------------------------------------------------------------------
+template <int D>
+__device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_wg, int lane, bool wait_select) {
+  constexpr int CH = D / 8;                   // 16-byte chunks per row
+  constexpr int KS = D / 16;
+  constexpr int NTL = D / 8;                  // 8-wide output tiles
+  constexpr int ROWB = D * 2;
+  constexpr int VOFF = 16 * ROWB;             // V half of a stage
+  constexpr int STAGE = 2 * VOFF;
+  constexpr int NCP = (16 * CH) / 32;         // cp.async per lane per operand per stage
+  const int gid = lane >> 2, tig = lane & 3;
+  const int G = p.G, L = p.L, P = p.P, units = p.B * p.Hkv, n_splits = p.n_splits;
+  const int gpb = L / 16;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(wsm);
+  uint32_t *goff = reinterpret_cast<uint32_t *>(wsm + kAttStages * kAttStageBytes);
+  int *gtok = reinterpret_cast<int *>(goff + kTableEntries);
+  const float sl2 = (1.0f / sqrtf((float)D)) * 1.4426950408889634f;
+  const uint4 *kbase = reinterpret_cast<const uint4 *>(p.k_pages) + lane;
+  const uint4 *vbase = reinterpret_cast<const uint4 *>(p.v_pages) + lane;
+
+  // lane-constant shared-memory offsets
+  uint32_t cdst[NCP];                          // destination of this lane's j-th 16-byte copy (swizzled)
+#pragma unroll
+  for (int j = 0; j < NCP; ++j) {
+    const int i = lane + 32 * j, t = i / CH, c = i - t * CH;
+    cdst[j] = t * ROWB + ((c ^ (t & 7)) << 4);
+  }
+  // ldmatrix row addresses.  K (not transposed): matrices (tokens 0-7, chunk 2s), (0-7, 2s+1), (8-15, 2s), (8-15, 2s+1)
+  const int kt = ((lane >> 4) & 1) * 8 + (lane & 7), kc = (lane >> 3) & 1;
+  // V (transposed): matrices (tokens 0-7, chunk 2np), (8-15, 2np), (0-7, 2np+1), (8-15, 2np+1)
+  const int vt = ((lane >> 3) & 1) * 8 + (lane & 7), vc = lane >> 4;
+
+  const long long n_items = (long long)units * n_splits;
+  for (long long item = wg; item < n_items; item += n_wg) {
+    const int u = (int)(item / n_splits), split = (int)(item - (long long)u * n_splits);
+    const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
+    const int T = p.seq_lens[b_idx];
+    const int ws = window_start(T, p.window, L);
+    const int n_cand = ws / L;
+    const int n_win = (T - ws + L - 1) / L;
+    int n_sel = min(p.topk, n_cand);
+    const int n_groups_u = (n_sel + n_win) * gpb;
+    const int per = (n_groups_u + n_splits - 1) / n_splits;
+    const int g0 = min(split * per, n_groups_u), g1 = min(g0 + per, n_groups_u);
+    int n_groups = min(g1 - g0, kTableEntries);
+    bool ok = true;
+    if (g0 < n_sel * gpb && n_groups > 0) {
+      if (wait_select) {
+        ok = wait_flag(p.ctl_ready + u);
+        if (!ok && lane == 0) report(p.status, COBS_ERR_TIMEOUT);
+        __threadfence();
+      } else {
+        n_sel = min(n_sel, min(__ldcg(p.sel_cnt + u), p.topk));
+      }
+    }
+    // ---- table of this item's groups -----------------------------------------------------------------
+    __syncwarp();
+    for (int g = lane; g < n_groups; g += 32) {
+      const int gg = g0 + g, it = gg / gpb, sub = gg - it * gpb;
+      int blk;
+      bool good = ok;
+      if (it < min(p.topk, n_cand)) {          // a selected-block slot
+        blk = (it < n_sel && ok) ? __ldcg(p.sel_idx + (size_t)u * p.topk + it) : -1;
+        if (it < n_sel && ok && (blk < 0 || blk >= n_cand)) { good = false; report(p.status, COBS_ERR_BOUNDS); }
+        if (blk < 0) good = false;
+      } else {
+        blk = n_cand + (it - min(p.topk, n_cand));
+      }
+      const int tok0 = blk * L + sub * 16;
+      int first = -1;
+      uint32_t off = 0;
+      if (good && tok0 < T) {
+        const int pg = p.page_table[(size_t)b_idx * p.mpp + tok0 / P];
+        if (pg < 0 || pg >= p.n_pages) report(p.status, COBS_ERR_BOUNDS);
+        else { first = tok0; off = (uint32_t)(((((size_t)pg * p.Hkv + h) * P + (tok0 % P)) * D) / 8); }
+      }
+      goff[g] = off;
+      gtok[g] = first;
+    }
+    __syncwarp();
+
+    // ---- query fragments: rows = heads (zero padded to 16), natural k order -----------------------------
+    uint32_t qa[KS][2];
+    {
+      const uint32_t *qg = reinterpret_cast<const uint32_t *>(p.q + ((size_t)b_idx * p.Hq + h * G + gid) * D);
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        qa[s][0] = (gid < G) ? qg[8 * s + tig] : 0u;
+        qa[s][1] = (gid < G) ? qg[8 * s + 4 + tig] : 0u;
+      }
+    }
+    float o[NTL][2];
+#pragma unroll
+    for (int n = 0; n < NTL; ++n) o[n][0] = o[n][1] = 0.f;
+    float m_run = -1e30f, l_run = 0.f, z2 = 0.f, z3 = 0.f;
+
+    auto issue = [&](int g, int st) {
+      if (g < n_groups) {
+        const int first = gtok[g];
+        if (first >= 0) {
+          const uint32_t off = goff[g];
+          const uint4 *ks = kbase + off, *vs = vbase + off;
+          const uint32_t dst = ring + st * STAGE;
+          const int nv = T - first;
+          if (nv >= 16) {
+#pragma unroll
+            for (int j = 0; j < NCP; ++j) { cpa16(dst + cdst[j], ks + 32 * j); cpa16(dst + VOFF + cdst[j], vs + 32 * j); }
+          } else {                             // ragged tail: rows past the end of the sequence are zero filled
+#pragma unroll
+            for (int j = 0; j < NCP; ++j) {
+              const int bytes = ((lane + 32 * j) / CH < nv) ? 16 : 0;
+              cpa16z(dst + cdst[j], ks + 32 * j, bytes);
+              cpa16z(dst + VOFF + cdst[j], vs + 32 * j, bytes);
+            }
+          }
+        }
+      }
+      cpa_commit();
+    };
+
+    issue(0, 0);
+    issue(1, 1);
+    int st = 0, st2 = 2;
+    for (int g = 0; g < n_groups; ++g) {
+      issue(g + 2, st2);
+      cpa_wait<2>();
+      __syncwarp();
+      const int first = gtok[g];
+      if (first >= 0) {
+        const uint32_t sb = ring + st * STAGE;
+        // ---- S^T = q K^T: s0 tokens 0-7, s1 tokens 8-15 --------------------------------------------------
+        float s00 = 0.f, s01 = 0.f, s10 = 0.f, s11 = 0.f;
+#pragma unroll
+        for (int s = 0; s < KS; ++s) {
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(b0, b1, b2, b3, sb + kt * ROWB + (((2 * s + kc) ^ (kt & 7)) << 4));
+          mma16816_bf16(s00, s01, z2, z3, qa[s][0], 0u, qa[s][1], 0u, b0, b1);
+          mma16816_bf16(s10, s11, z2, z3, qa[s][0], 0u, qa[s][1], 0u, b2, b3);
+        }
+        const int nv = T - first;
+        if (nv < 16) {                         // tokens past the end take no weight
+          if (2 * tig >= nv) s00 = -1e30f;
+          if (2 * tig + 1 >= nv) s01 = -1e30f;
+          if (2 * tig + 8 >= nv) s10 = -1e30f;
+          if (2 * tig + 9 >= nv) s11 = -1e30f;
+        }
+        float mx = fmaxf(fmaxf(s00, s01), fmaxf(s10, s11));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        if (__any_sync(0xffffffffu, mx > m_run)) {       // rescale only when some head's running max moved
+          const float m_new = fmaxf(m_run, mx);
+          const float corr = ex2((m_run - m_new) * sl2);
+          m_run = m_new;
+          l_run *= corr;
+#pragma unroll
+          for (int n = 0; n < NTL; ++n) { o[n][0] *= corr; o[n][1] *= corr; }
+        }
+        const float mb = m_run * sl2;
+        const float p0 = ex2(fmaf(s00, sl2, -mb)), p1 = ex2(fmaf(s01, sl2, -mb));
+        const float p2 = ex2(fmaf(s10, sl2, -mb)), p3 = ex2(fmaf(s11, sl2, -mb));
+        l_run += (p0 + p1) + (p2 + p3);
+        const uint32_t a0h = bf16x2(p0, p1), a2h = bf16x2(p2, p3);
+        const uint32_t a0l = bf16x2(p0 - bf16_lo(a0h), p1 - bf16_hi(a0h));
+        const uint32_t a2l = bf16x2(p2 - bf16_lo(a2h), p3 - bf16_hi(a2h));
+        // ---- O += P V ---------------------------------------------------------------------------------------
+#pragma unroll
+        for (int np = 0; np < NTL / 2; ++np) {
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(b0, b1, b2, b3, sb + VOFF + vt * ROWB + (((2 * np + vc) ^ (vt & 7)) << 4));
+          mma16816_bf16(o[2 * np][0], o[2 * np][1], z2, z3, a0h, 0u, a2h, 0u, b0, b1);
+          mma16816_bf16(o[2 * np + 1][0], o[2 * np + 1][1], z2, z3, a0h, 0u, a2h, 0u, b2, b3);
+          mma16816_bf16(o[2 * np][0], o[2 * np][1], z2, z3, a0l, 0u, a2l, 0u, b0, b1);
+          mma16816_bf16(o[2 * np + 1][0], o[2 * np + 1][1], z2, z3, a0l, 0u, a2l, 0u, b2, b3);
+        }
+      }
+      __syncwarp();                            // all lanes are done with the stage before it is refilled
+      st = (st == kAttStages - 1) ? 0 : st + 1;
+      st2 = (st2 == kAttStages - 1) ? 0 : st2 + 1;
+    }
+    cpa_wait<0>();
+
+    // ---- this warp's partial: [G][D + 2] = acc, running max (natural log units), running sum ----------------
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    float *part = p.partial + ((size_t)u * n_splits + split) * G * (D + 2);
+    if (gid < G) {
+      float *dst = part + gid * (D + 2);
+#pragma unroll
+      for (int n = 0; n < NTL; ++n) __stcg(reinterpret_cast<float2 *>(dst + 8 * n + 2 * tig), make_float2(o[n][0], o[n][1]));
+      if (tig == 0) {
+        __stcg(dst + D, (l_run > 0.f) ? m_run * (sl2 * 0.6931471805599453f) : -INFINITY);
+        __stcg(dst + D + 1, l_run);
+      }
+    }
+    __threadfence();
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) last = (atomicAdd(p.ctl_att + u, 1) + 1 == n_splits);
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (last) {
+      // ---- merge the unit's partials: o = sum_s e^{m_s - M} acc_s / sum_s e^{m_s - M} l_s -------------------
+      __threadfence();
+      const float *pu = p.partial + (size_t)u * n_splits * G * (D + 2);
+      for (int g = 0; g < G; ++g) {
+        float M = -INFINITY;
+        for (int s = 0; s < n_splits; ++s) M = fmaxf(M, __ldcg(pu + ((size_t)s * G + g) * (D + 2) + D));
+        float den = 0.f;
+        float acc[D / 32];
+#pragma unroll
+        for (int k = 0; k < D / 32; ++k) acc[k] = 0.f;
+        for (int s = 0; s < n_splits; ++s) {
+          const float *ps = pu + ((size_t)s * G + g) * (D + 2);
+          const float m = __ldcg(ps + D);
+          const float w = (m == -INFINITY) ? 0.f : __expf(m - M);
+          den = fmaf(w, __ldcg(ps + D + 1), den);
+#pragma unroll
+          for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(w, __ldcg(ps + lane + 32 * k), acc[k]);
+        }
+        const size_t bh = (size_t)b_idx * p.Hq + h * G + g;
+#pragma unroll
+        for (int k = 0; k < D / 32; ++k) p.out[bh * D + lane + 32 * k] = acc[k] / den;
+        if (p.lse && lane == 0) p.lse[bh] = M + logf(den);
+      }
+    }
+    __syncwarp();
+  }
+}
+
+#ifdef COBS_TIMING
+// development aid: per-warp phase boundary timestamps (ns), read back by cobs_debug_times
+__device__ unsigned long long g_dbg_times[4][4096];
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define COBS_STAMP(k) do { if (lane == 0 && wg < 4096) g_dbg_times[k][wg] = gtime(); } while (0)
+#else
+#define COBS_STAMP(k) do { } while (0)
+#endif
+
+// ---------------------------------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------------------------------
+template <int DT, int D, int WPT, int NT>
+__global__ void __launch_bounds__(kFThreads, 2) fused_step_kernel(Params p, int phases) {
+  extern __shared__ __align__(256) unsigned char fsm[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wg = blockIdx.x * kFWarps + warp, n_wg = gridDim.x * kFWarps;
+  unsigned char *wsm = fsm + warp * kWarpSmemBytes;
+  COBS_STAMP(0);
+  if (phases & PH_SCORE) {
+    score_phase<DT, D, WPT, NT>(p, wsm, wg, n_wg, lane);
+    COBS_STAMP(1);
+    __syncthreads();                       // the four rings are idle: the selection uses them as one scratch area
+    select_phase(p, fsm);
+    __syncthreads();
+  }
+  COBS_STAMP(2);
+  if (phases & PH_ATTEND) attend_phase<D>(p, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
+  COBS_STAMP(3);
+  // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
+  __syncthreads();
+  __shared__ int is_last;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    is_last = (atomicAdd(p.ctl_done, 1) + 1 == (int)gridDim.x);
+  }
+  __syncthreads();
+  if (is_last) {
+    const int units = p.B * p.Hkv;
+    for (int i = threadIdx.x; i < units; i += kFThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
+    if (threadIdx.x == 0) *p.ctl_done = 0;
+  }
+}
+
+// q~ = U_Q^T (q / sqrt(D)) for every query head, zero padded to Ds_pad (subspace descriptor only).
+__global__ void qtilde_kernel(Params p) {
+  const int bh = blockIdx.x, b_idx = bh / p.Hq, hq = bh - b_idx * p.Hq, h = hq / p.G;
+  extern __shared__ float qs[];
+  const float inv_sqrt_d = 1.0f / sqrtf((float)p.D);
+  for (int d = threadIdx.x; d < p.D; d += blockDim.x) qs[d] = __bfloat162float(p.q[(size_t)bh * p.D + d]) * inv_sqrt_d;
+  __syncthreads();
+  for (int s = threadIdx.x; s < p.Ds_pad; s += blockDim.x) {
+    float v = 0.f;
+    if (s < p.Ds) {
+      const float *uq = p.u_q + (size_t)h * p.D * p.Ds + s;
+      for (int d = 0; d < p.D; ++d) v = fmaf(uq[(size_t)d * p.Ds], qs[d], v);
+    }
+    p.qtilde_out[(size_t)bh * p.Ds_pad + s] = v;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------------
+template <int DT, int D, int WPT, int NT>
+static cudaError_t launch_fused_t(Params p, int phases, cudaStream_t stream) {
+  auto kern = fused_step_kernel<DT, D, WPT, NT>;
+  static int grid_cache[64] = {0};             // resident grid size of this instantiation, per device
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (grid_cache[dev] == 0) {
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBytes)) != cudaSuccess) return e;
+    int sms = 0, occ = 0;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kFThreads, kFusedSmemBytes)) != cudaSuccess) return e;
+    if (occ < 1) return cudaErrorLaunchOutOfResources;
+    grid_cache[dev] = sms * occ;
+  }
+  void *args[] = {&p, &phases};
+  // cooperative launch: the grid is resident as a whole (or the launch fails), which the cross-warp waits rely on
+  e = cudaLaunchCooperativeKernel((const void *)kern, dim3(grid_cache[dev]), dim3(kFThreads), args, kFusedSmemBytes,
+                                  stream);
+  count_launch();
+  return e;
+}
+
+// Whether the persistent kernel covers this configuration's scoring phase.
+bool fused_score_supported(const Params &p) {
+  if (p.NB > kMaxSelectBlocks) return false;
+  if (p.summ_dtype == COBS_SUMM_BF16) return p.u_q == nullptr;
+  if (p.summ_dtype == COBS_SUMM_FP4_E2M1) {
+    if (p.Ds_pad % 32 != 0) return false;
+    const int scale_sz = (p.scale_dtype == COBS_SCALE_FP16) ? 2 : 4;
+    if ((p.r * scale_sz) % 4 != 0) return false;
+    return true;
+  }
+  return false;
+}
+
+cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream) {
+  if ((phases & PH_SCORE) && p.u_q) {
+    Params q = p;
+    qtilde_kernel<<<p.B * p.Hq, 128, p.D * sizeof(float), stream>>>(q);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  const bool fp4 = p.summ_dtype == COBS_SUMM_FP4_E2M1 && (phases & PH_SCORE);
+  if (!fp4) {
+    return p.D == 128 ? launch_fused_t<COBS_SUMM_BF16, 128, 1, 1>(p, phases, stream)
+                      : launch_fused_t<COBS_SUMM_BF16, 64, 1, 1>(p, phases, stream);
+  }
+  const int wpt = p.Ds_pad / 32;
+  const bool sub = p.u_q != nullptr;
+#define COBS_CASE(DD, WW)                                                                                   \
+  if (p.D == DD && wpt == WW)                                                                               \
+    return sub ? launch_fused_t<COBS_SUMM_FP4_E2M1, DD, WW, 2>(p, phases, stream)                           \
+               : launch_fused_t<COBS_SUMM_FP4_E2M1, DD, WW, 1>(p, phases, stream);
+  COBS_CASE(128, 4) COBS_CASE(128, 3) COBS_CASE(128, 2) COBS_CASE(128, 1) COBS_CASE(64, 2) COBS_CASE(64, 1)
+#undef COBS_CASE
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace cobs
+
+#ifdef COBS_TIMING
+extern "C" int cobs_debug_times(unsigned long long *host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_times, sizeof(unsigned long long) * 4 * 4096);
+}
+#endif

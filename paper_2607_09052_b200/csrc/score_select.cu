@@ -279,12 +279,7 @@ static cudaError_t launch_score_g(const Params &p, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_score_fast(const Params &p, cudaStream_t stream, bool *handled);
-
 cudaError_t launch_score(const Params &p, cudaStream_t stream) {
-  bool handled = false;
-  cudaError_t e = launch_score_fast(p, stream, &handled);
-  if (handled || e != cudaSuccess) return e;
   switch (p.G) {
     case 1: return launch_score_g<1>(p, stream);
     case 2: return launch_score_g<2>(p, stream);
