@@ -59,6 +59,8 @@ static int32_t validate_config(const cobs_config *c) {
   // an attention slice holds at most kItemGroups 16-token groups and a unit at most kMaxSplits slices
   if ((long long)max_items(c) * (c->block_size / 16) > (long long)kItemGroups * kMaxSplits) return COBS_ERR_UNSUPPORTED;
   if ((long long)c->batch * c->n_kv_heads > kMaxUnits) return COBS_ERR_UNSUPPORTED;
+  // chunk and item indices are 32-bit
+  if ((long long)c->batch * c->n_kv_heads * ((c->max_blocks + 15) / 16) > 0x3fffffffLL) return COBS_ERR_UNSUPPORTED;
   return COBS_OK;
 }
 

@@ -40,21 +40,39 @@ namespace cobs {
 
 constexpr int kFWarps = 4;
 constexpr int kFThreads = kFWarps * 32;
-constexpr int kSlots = 24;                                   // 16-byte slots per lane per scoring stage
-constexpr int kScaleBytes = 16 * COBS_MAX_RANK * 4;          // scales of a chunk (16 blocks x r, fp32)
-constexpr int kScoreStageBytes = kSlots * 512 + kScaleBytes; // 13312
+constexpr int kScoreStageBytes = 14080;                      // means + factor rows + scales of a 16-block chunk
 constexpr int kAttStages = 3;
 constexpr int kAttStageBytes = 2 * 16 * 128 * 2;             // K + V of one 16-token group, D = 128
-constexpr int kHistBytes = 1024;
 constexpr int kTableEntries = 256;                           // 16-token groups per attention item
 constexpr int kRingBytes = (2 * kScoreStageBytes > kAttStages * kAttStageBytes + kTableEntries * 8)
                                ? 2 * kScoreStageBytes : kAttStages * kAttStageBytes + kTableEntries * 8;
-constexpr int kWarpSmemBytes = kRingBytes + kHistBytes;      // 27648
-constexpr int kFusedSmemBytes = kFWarps * kWarpSmemBytes;    // 110592
+constexpr int kWarpSmemBytes = kRingBytes;                   // 28160
+constexpr int kFusedSmemBytes = kFWarps * kWarpSmemBytes;    // 112640: two CTAs per SM
 constexpr int kMaxSelectBlocks = 16384;                      // scores + chunk weights of a unit fit the CTA's shared memory
 constexpr long long kSpinLimit = 4000000;                    // x ~100 ns: bounded wait on another warp
 
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
+
+#ifdef COBS_TIMING
+// development aid: per-warp phase boundary timestamps (ns), read back by cobs_debug_times
+__device__ unsigned long long g_dbg_times[4][4096];
+__device__ unsigned long long g_dbg_acc[8][4096];   // per-warp accumulated clock cycles by category
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define COBS_STAMP(k) do { if (lane == 0 && wg < 4096) g_dbg_times[k][wg] = gtime(); } while (0)
+#define COBS_ACC_DECL long long acc_t[8] = {0,0,0,0,0,0,0,0}; long long acc_last = clock64()
+#define COBS_ACC(k) do { long long now_ = clock64(); acc_t[k] += now_ - acc_last; acc_last = now_; } while (0)
+#define COBS_ACC_FLUSH(id) do { if ((threadIdx.x & 31) == 0 && (id) < 4096) { for (int k_ = 0; k_ < 8; ++k_) g_dbg_acc[k_][id] += acc_t[k_]; } } while (0)
+#else
+#define COBS_ACC_DECL do { } while (0)
+#define COBS_ACC(k) do { } while (0)
+#define COBS_ACC_FLUSH(id) do { } while (0)
+#define COBS_STAMP(k) do { } while (0)
+#endif
+
 
 // ---------------------------------------------------------------------------------------------------
 // small PTX helpers
@@ -121,6 +139,33 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+  return v;
+}
+// ---- mbarrier + bulk copy (global -> shared, completion counted in bytes on an mbarrier) -----------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Wait for the phase with the given parity to complete.  Bounded; false on expiry.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (int it = 0; it < 20000000; ++it) {
+    uint32_t done;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
 }
 __device__ __forceinline__ int ld_volatile(const int *p) { return *reinterpret_cast<const volatile int *>(p); }
 
@@ -193,12 +238,18 @@ __device__ void select_phase(const Params &p, unsigned char *cta_smem) {
     if (!s_ok) { __syncthreads(); continue; }                  // never scored: leave the unit unselected
     __threadfence();
 
-    // ---- lse per head from the chunk pairs ------------------------------------------------------------
+    // ---- chunk pairs -> shared memory (one L2 round trip), lse per head -------------------------------------
     const float2 *pp = reinterpret_cast<const float2 *>(p.lse_part) + (size_t)u * G * cpu;
+    float2 *pairs = reinterpret_cast<float2 *>(cw + 8 * cpu);   // [G][chunks]
+    for (int i = tid; i < G * n_chunks; i += kFThreads) {
+      const int g = i / n_chunks, c = i - g * n_chunks;
+      pairs[g * cpu + c] = __ldcg(pp + (size_t)g * cpu + c);
+    }
+    __syncthreads();
     for (int g = 0; g < G; ++g) {
       float m = -INFINITY, s = 0.f;
       for (int c = tid; c < n_chunks; c += kFThreads) {
-        const float2 v = __ldcg(pp + (size_t)g * cpu + c);
+        const float2 v = pairs[g * cpu + c];
         const float nm = fmaxf(m, v.x);
         s = s * expf(m - nm) + v.y * expf(v.x - nm);
         m = nm;
@@ -223,22 +274,22 @@ __device__ void select_phase(const Params &p, unsigned char *cta_smem) {
     __syncthreads();
     for (int i = tid; i < G * n_chunks; i += kFThreads) {
       const int g = i / n_chunks, c = i - g * n_chunks;
-      cw[g * cpu + c] = expf(__ldcg(pp + (size_t)g * cpu + c).x - s_lse[g]);
+      cw[g * cpu + c] = expf(pairs[g * cpu + c].x - s_lse[g]);
     }
     __syncthreads();
-    // ---- scores -------------------------------------------------------------------------------------------
+    // ---- scores: t values from L2, eight per head per thread in flight ------------------------------------------
     const float *tu = p.e + (size_t)u * G * NB;
-    for (int b0 = 0; b0 < n_sum; b0 += 4 * kFThreads) {
-      float x[8][4];
+    for (int b0 = 0; b0 < n_sum; b0 += 8 * kFThreads) {
+      float x[8][8];
 #pragma unroll
       for (int g = 0; g < 8; ++g)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 8; ++j) {
           const int b = b0 + tid + kFThreads * j;
           x[g][j] = (g < G && b < n_sum) ? __ldcg(tu + (size_t)g * NB + b) : 0.f;
         }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < 8; ++j) {
         const int b = b0 + tid + kFThreads * j;
         if (b < n_sum) {
           float sv = 0.f;
@@ -335,122 +386,141 @@ __device__ void select_phase(const Params &p, unsigned char *cta_smem) {
 // (Ds_pad / 32).  NT: f16 terms of the query (1: full space, 2: fp32 subspace query).
 // ---------------------------------------------------------------------------------------------------
 template <int DT, int D, int WPT, int NT>
-__device__ void score_phase(const Params &p, unsigned char *wsm, int wg, int n_wg, int lane) {
+__device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars, int wg, int n_wg, int lane) {
   constexpr bool FP4 = (DT == COBS_SUMM_FP4_E2M1);
   constexpr int MCH = D / 32;                 // 16-byte chunks of a bf16 row per thread
-  constexpr int MEAN_SLOTS = 2 * MCH;         // two blocks
-  constexpr int ROW_SLOTS = FP4 ? 2 : 2 * MCH;
-  constexpr int ROWS0 = (kSlots - MEAN_SLOTS) / ROW_SLOTS;   // factor rows that fit beside the means
-  constexpr int ROWSN = kSlots / ROW_SLOTS;                  // factor rows of a later batch
   constexpr int KSM = D / 16;                 // k-steps of a bf16 row
   constexpr int KSQ = FP4 ? WPT * 2 : 1;      // k-steps of an FP4 row
+  // stage layout: [16 block means, row stride MROW][16 blocks x rows of factors, block stride XS][scales]
+  // The +32 bytes of padding per row / block put the rows of neighbouring quads in different bank halves.
+  constexpr int MROW = D * 2 + 32;
+  constexpr int MEAN_BYTES = 16 * MROW;
+  constexpr int ROWB = FP4 ? WPT * 16 : D * 2;                 // bytes of one factor row
+  constexpr int ROWS_CAP = (kScoreStageBytes - 16 * 32) / (16 * ROWB);
+  constexpr int ROWS_MAX = ROWS_CAP < COBS_MAX_RANK ? ROWS_CAP : COBS_MAX_RANK;   // rows a batch can hold at most
+  static_assert((kScoreStageBytes - MEAN_BYTES - 16 * 32 - 16 * COBS_MAX_RANK * 4) / (16 * ROWB) >= 1, "stage too small");
   const int gid = lane >> 2, tig = lane & 3;
   const int G = p.G, r = p.r, NB = p.NB, L = p.L;
   const int units = p.B * p.Hkv;
   const int cpu = (NB + 15) / 16;             // chunks per unit
-  const long long total = (long long)units * cpu;
+  const int scale_sz = (p.scale_dtype == COBS_SCALE_FP16) ? 2 : 4;
+  const int scale_bytes = FP4 ? 16 * r * scale_sz : 0;        // scales of a chunk, at the end of the stage
+  // Common case: means, all r factor rows and scales of the 16 blocks fit one stage.  Then a chunk is three
+  // contiguous pieces of the summary arrays and is fetched by three bulk copies in memory layout (`single`).
+  // Otherwise the factor rows go in batches, each block copied on its own to a padded position.
+  const bool single = 16 * D * 2 + 16 * r * ROWB + scale_bytes <= kScoreStageBytes && r <= ROWS_MAX;
+  const int ROWS0 = single ? r : min(ROWS_MAX, (kScoreStageBytes - MEAN_BYTES - 16 * 32 - scale_bytes) / (16 * ROWB));
+  const int ROWSN = min(ROWS_MAX, (kScoreStageBytes - 16 * 32 - scale_bytes) / (16 * ROWB));
+  const int mrow = single ? D * 2 : MROW;                                  // row stride of the mean area
+  const int mean_bytes = 16 * mrow;
+  const int XS0 = single ? r * ROWB : ROWS0 * ROWB + 32, XSN = ROWSN * ROWB + 32;   // block stride of the factor area
   const int n_batches = (r <= ROWS0) ? 1 : 1 + (r - ROWS0 + ROWSN - 1) / ROWSN;
   const uint32_t ring = (uint32_t)__cvta_generic_to_shared(wsm);
+  const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
   const float inv_sqrt_d = 1.0f / sqrtf((float)D);
   const float ln_l = logf((float)L);
-  const int row_bytes = FP4 ? p.Ds_pad / 2 : D * 2;
-  const int scale_sz = (p.scale_dtype == COBS_SCALE_FP16) ? 2 : 4;
 
-  // position in this warp's batch sequence: chunk c (global index), batch b
-  auto chunk_valid = [&](long long c, int &u, int &n_sum) -> bool {
-    if (c >= total) return false;
-    u = (int)(c / cpu);
-    n_sum = min(p.seq_lens[u / p.Hkv] / L, NB);
-    const int ck = (int)(c - (long long)u * cpu);
-    // chunk 0 of a unit without summarised blocks is still visited: its warp publishes the empty selection
-    return ck * 16 < n_sum || ck == 0;
-  };
-  // this warp's contiguous range of chunks (mostly one unit: its query fragments are built once)
-  const long long per_warp = (total + n_wg - 1) / n_wg;
-  const long long c_begin = min((long long)wg * per_warp, total), c_end = min(c_begin + per_warp, total);
-  auto next_chunk = [&](long long c) -> long long {
-    int u, n;
-    while (c < c_end && !chunk_valid(c, u, n)) c = (long long)(u + 1) * cpu;   // rest of the unit has no summaries
-    return c < c_end ? c : total;
-  };
-
-  // ---- issue the copies of (chunk c, batch b) into stage st -----------------------------------------
-  auto issue = [&](long long c, int b, int st) {
-    if (c < total) {
-      const int u = (int)(c / cpu), ck = (int)(c - (long long)u * cpu);
+  // This warp's contiguous range of chunks (mostly one unit: its query fragments are built once).
+  // Positions are (unit, chunk-in-unit) pairs advanced incrementally; 32-bit arithmetic throughout.
+  const int total = units * cpu;              // the host refuses configurations where this overflows
+  const int per_warp = (total + n_wg - 1) / n_wg;
+  const int c_begin = min(wg * per_warp, total), c_end = min(c_begin + per_warp, total);
+  // first position at or after (u, ck) that holds work, or u = units when the range is exhausted.
+  // Chunk 0 of a unit without summarised blocks counts as work: its warp counts it, so that the
+  // selection phase sees the unit as scored.
+  auto seek = [&](int &u, int &ck) {
+    while (u < units && u * cpu + ck < c_end) {
       const int n_sum = min(p.seq_lens[u / p.Hkv] / L, NB);
-      if (ck * 16 < n_sum) {
-        const int bA = min(ck * 16 + 2 * gid, NB - 1), bB = min(ck * 16 + 2 * gid + 1, NB - 1);
-        const size_t rec[2] = {(size_t)u * NB + bA, (size_t)u * NB + bB};
-        const uint32_t base = ring + st * kScoreStageBytes + lane * 16;
-        int slot = 0;
-        if (b == 0) {
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            const char *src = (const char *)p.mean + rec[a] * (size_t)(D * 2) + tig * 16;
-#pragma unroll
-            for (int m = 0; m < MCH; ++m) cpa16(base + (a * MCH + m) * 512, src + m * 64);
-          }
-          slot = MEAN_SLOTS;
-        }
-        if (FP4) {        // scales of the two blocks of this quad (every batch: a batch may sit in either stage)
-          const uint32_t sbase = ring + st * kScoreStageBytes + kSlots * 512;
-          const int per_blk = r * scale_sz;                    // bytes per block, a multiple of 4
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            const char *src = (const char *)p.scale + rec[a] * (size_t)per_blk;
-            for (int w = tig * 4; w < per_blk; w += 16) cpa4(sbase + (2 * gid + a) * 64 + w, src + w);
-          }
-        }
-        const int row0 = (b == 0) ? 0 : ROWS0 + (b - 1) * ROWSN;
-        const int rows = min(r - row0, (b == 0) ? ROWS0 : ROWSN);
-        for (int i = 0; i < rows; ++i) {
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            const char *src = (const char *)p.xi + (rec[a] * r + row0 + i) * (size_t)row_bytes;
-            if (FP4) {
-              const uint32_t dst = base + (slot + i * 2 + a) * 512;
-              if (WPT == 4) cpa16(dst, src + tig * 16);
-              else {
-#pragma unroll
-                for (int w = 0; w < WPT; ++w) cpa4(dst + w * 4, src + (tig * WPT + w) * 4);
-              }
-            } else {
-#pragma unroll
-              for (int m = 0; m < MCH; ++m) cpa16(base + (slot + (i * 2 + a) * MCH + m) * 512, src + tig * 16 + m * 64);
-            }
-          }
-        }
+      if (ck * 16 < n_sum || ck == 0) return;
+      ++u; ck = 0;                             // rest of this unit has no summaries
+    }
+    u = units;
+  };
+
+  // ---- bulk copies of (chunk c, batch b) into stage st; completion is counted on the stage's mbarrier ----
+  // lanes 0-15 copy the factor rows of block `lane`, lanes 16-31 the mean of block `lane - 16`, lane 0 the scales
+  auto issue = [&](int u, int ck, int b, int st) {
+    if (u >= units) return;
+    const int n_sum = min(p.seq_lens[u / p.Hkv] / L, NB);
+    if (ck * 16 >= n_sum) return;
+    const int nblk = min(16, NB - ck * 16);
+    const size_t rec0 = (size_t)u * NB + ck * 16;
+    const int row0 = (b == 0) ? 0 : ROWS0 + (b - 1) * ROWSN;
+    const int rows = min(r - row0, (b == 0) ? ROWS0 : ROWSN);
+    const uint32_t sbase = ring + st * kScoreStageBytes;
+    const uint32_t xoff = (b == 0) ? mean_bytes : 0;
+    const uint32_t xs = (b == 0) ? XS0 : XSN;
+    const uint32_t soff = kScoreStageBytes - scale_bytes;
+    const bool scales_bulk = FP4 && nblk == 16 && r > 0;
+    const uint32_t bar = bar0 + st * 8;
+    if (lane == 0) {
+      uint32_t tx = (uint32_t)nblk * (uint32_t)(rows > 0 ? rows * ROWB : 0);
+      if (b == 0) tx += (uint32_t)nblk * (D * 2);
+      if (scales_bulk) tx += (uint32_t)(16 * r * scale_sz);
+      fence_proxy_async();
+      mbar_expect_tx(bar, tx);
+    }
+    __syncwarp();
+    if (single) {
+      if (lane == 0) bulk_g2s(sbase, (const char *)p.mean + rec0 * (size_t)(D * 2), nblk * D * 2, bar);
+      if (lane == 1 && rows > 0) bulk_g2s(sbase + xoff, (const char *)p.xi + rec0 * r * (size_t)ROWB, nblk * r * ROWB, bar);
+    } else if (lane < 16) {
+      if (lane < nblk && rows > 0)
+        bulk_g2s(sbase + xoff + lane * xs, (const char *)p.xi + ((rec0 + lane) * r + row0) * (size_t)ROWB, rows * ROWB, bar);
+    } else if (b == 0 && lane - 16 < nblk) {
+      bulk_g2s(sbase + (lane - 16) * mrow, (const char *)p.mean + (rec0 + lane - 16) * (size_t)(D * 2), D * 2, bar);
+    }
+    if (FP4 && r > 0) {
+      const char *ssrc = (const char *)p.scale + rec0 * (size_t)(r * scale_sz);
+      if (scales_bulk) {
+        if (lane == 2) bulk_g2s(sbase + soff, ssrc, 16 * r * scale_sz, bar);
+      } else {                                // ragged last chunk of the array: plain loads, 4 bytes at a time
+        for (int w = lane * 4; w < nblk * r * scale_sz; w += 128)
+          *reinterpret_cast<uint32_t *>(wsm + st * kScoreStageBytes + soff + w) = *reinterpret_cast<const uint32_t *>(ssrc + w);
       }
     }
-    cpa_commit();
   };
 
-  long long cur = next_chunk(c_begin);
+  int cu = c_begin / cpu, cck = c_begin - cu * cpu;        // current position
+  if (c_begin >= c_end) cu = units; else seek(cu, cck);
   int cur_b = 0, st = 0;
+  uint32_t phase_bits = 0;                  // bit st = parity to wait for on stage st
   int pend_u = -1, pend_n = 0;              // chunks finished but not yet counted (counted once per unit run)
-  issue(cur, 0, 0);
+  issue(cu, cck, 0, 0);
   // per-chunk state
   uint32_t bm[KSM][2];
   uint32_t bq[FP4 ? NT : 1][KSQ][2];
   float m0 = 0.f, m1 = 0.f;
   float fA0 = 0.f, fA1 = 0.f, fB0 = 0.f, fB1 = 0.f, sA0 = 0.f, sA1 = 0.f, sB0 = 0.f, sB1 = 0.f;
   int cur_u = -1;
+  bool alive = true;
 
-  while (cur < total) {
+  COBS_ACC_DECL;
+  while (cu < units && alive) {
+    COBS_ACC(0);
     // ---- prefetch the next batch of this warp --------------------------------------------------------
-    long long nxt = cur;
-    int nxt_b = cur_b + 1;
-    if (nxt_b >= n_batches) { nxt_b = 0; nxt = next_chunk(cur + 1); }
-    issue(nxt, nxt_b, st ^ 1);
-    cpa_wait<1>();
-    __syncwarp();
+    int nu = cu, nck = cck, nxt_b = cur_b + 1;
+    if (nxt_b >= n_batches) {
+      nxt_b = 0;
+      if (++nck >= cpu) { ++nu; nck = 0; }
+      seek(nu, nck);
+    }
+    issue(nu, nck, nxt_b, st ^ 1);
+    COBS_ACC(1);
 
-    const int u = (int)(cur / cpu), ck = (int)(cur - (long long)u * cpu);
+    const int u = cu, ck = cck;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
     const int n_sum = min(p.seq_lens[b_idx] / L, NB);
-    const uint32_t base = ring + st * kScoreStageBytes + lane * 16;
+    const uint32_t sbase = ring + st * kScoreStageBytes;
     if (ck * 16 < n_sum) {
+      if (!mbar_wait(bar0 + st * 8, (phase_bits >> st) & 1u)) {     // bounded: the copies never landed
+        if (lane == 0) report(p.status, COBS_ERR_TIMEOUT);
+        alive = false;
+        break;
+      }
+      phase_bits ^= 1u << st;
+      __syncwarp();
+      COBS_ACC(2);
       if (cur_b == 0) {
         if (u != cur_u) {
           cur_u = u;
@@ -469,17 +539,21 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, int wg, int n_w
             float mx = 0.f;
 #pragma unroll
             for (int j = 0; j < WPT; ++j) {
-#pragma unroll
-              for (int n = 0; n < 8; ++n) {
-                float v = 0.f;
-                const int idx = tig * (WPT * 8) + j * 8 + n;
-                if (gid < G) {
-                  if (p.qtilde) v = p.qtilde[((size_t)b_idx * p.Hq + h * G + gid) * p.Ds_pad + idx];
-                  else v = __bfloat162float(qg[gid * D + idx]);
-                }
-                e[j][n] = v;
-                mx = fmaxf(mx, fabsf(v));
+              if (p.qtilde) {
+                const float4 *src = reinterpret_cast<const float4 *>(
+                    p.qtilde + ((size_t)b_idx * p.Hq + h * G + gid) * p.Ds_pad + tig * (WPT * 8) + j * 8);
+                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+                if (gid < G) { lo = src[0]; hi = src[1]; }
+                e[j][0] = lo.x; e[j][1] = lo.y; e[j][2] = lo.z; e[j][3] = lo.w;
+                e[j][4] = hi.x; e[j][5] = hi.y; e[j][6] = hi.z; e[j][7] = hi.w;
+              } else {
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (gid < G) v = *reinterpret_cast<const uint4 *>(qg + gid * D + tig * (WPT * 8) + j * 8);
+                e[j][0] = bf16_lo(v.x); e[j][1] = bf16_hi(v.x); e[j][2] = bf16_lo(v.y); e[j][3] = bf16_hi(v.y);
+                e[j][4] = bf16_lo(v.z); e[j][5] = bf16_hi(v.z); e[j][6] = bf16_lo(v.w); e[j][7] = bf16_hi(v.w);
               }
+#pragma unroll
+              for (int n = 0; n < 8; ++n) mx = fmaxf(mx, fabsf(e[j][n]));
             }
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
@@ -494,23 +568,25 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, int wg, int n_w
                 float hi[8];
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
-                  hi[n] = __half2float(__float2half_rn(e[j][n] * (t == 0 ? inv_s : 1.0f)));
-                  e[j][n] = e[j][n] * (t == 0 ? inv_s : 1.0f) - hi[n];
+                  const float x = (t == 0) ? e[j][n] * inv_s : e[j][n];
+                  hi[n] = __half2float(__float2half_rn(x));
+                  e[j][n] = x - hi[n];
                 }
                 bq[t][2 * j][0] = f16x2(hi[0], hi[1]); bq[t][2 * j][1] = f16x2(hi[2], hi[3]);
                 bq[t][2 * j + 1][0] = f16x2(hi[4], hi[5]); bq[t][2 * j + 1][1] = f16x2(hi[6], hi[7]);
               }
             }
-            // head 2 tig, 2 tig + 1 of the result columns belong to the lanes gid = 2 tig, 2 tig + 1 of any quad
+            // result columns 2 tig, 2 tig + 1 are heads whose factor sits in the lanes gid = 2 tig, 2 tig + 1
             m0 = __shfl_sync(0xffffffffu, mult, (2 * tig) * 4);
             m1 = __shfl_sync(0xffffffffu, mult, (2 * tig + 1) * 4);
           }
         }
         // ---- first-order term: block means against the raw bf16 query ------------------------------------
         float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+        const uint32_t ma = sbase + (2 * gid) * mrow + tig * 16, mb = ma + mrow;
 #pragma unroll
         for (int m = 0; m < MCH; ++m) {
-          const uint4 va = lds128(base + m * 512), vb = lds128(base + (MCH + m) * 512);
+          const uint4 va = lds128(ma + m * 64), vb = lds128(mb + m * 64);
           mma16816_bf16(c0, c1, c2, c3, va.x, vb.x, va.y, vb.y, bm[2 * m][0], bm[2 * m][1]);
           mma16816_bf16(c0, c1, c2, c3, va.z, vb.z, va.w, vb.w, bm[2 * m + 1][0], bm[2 * m + 1][1]);
         }
@@ -518,61 +594,90 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, int wg, int n_w
         sA0 = sA1 = sB0 = sB1 = 0.f;
       }
       // ---- curvature term: rows of this batch ----------------------------------------------------------
-      const int slot0 = (cur_b == 0) ? MEAN_SLOTS : 0;
       const int row0 = (cur_b == 0) ? 0 : ROWS0 + (cur_b - 1) * ROWSN;
       const int rows = min(r - row0, (cur_b == 0) ? ROWS0 : ROWSN);
-      const uint32_t sbase = ring + st * kScoreStageBytes + kSlots * 512 + (2 * gid) * 64;
+      const uint32_t xs = (cur_b == 0) ? XS0 : XSN;
+      const uint32_t xa = sbase + ((cur_b == 0) ? mean_bytes : 0) + (2 * gid) * xs + tig * (FP4 ? WPT * 4 : 16), xb = xa + xs;
+      if (FP4) {
+        // four factor rows at a time: four independent accumulator chains keep the tensor pipe busy
+        constexpr int RG = 4;
+        const unsigned char *sp = wsm + st * kScoreStageBytes + (kScoreStageBytes - scale_bytes) + (2 * gid) * r * scale_sz;
 #pragma unroll
-      for (int i = 0; i < ROWSN; ++i) {
-        if (i < rows) {
-          float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-          if (FP4) {
-            uint32_t wa[4], wb[4];
-            if (WPT == 4) {
-              const uint4 a = lds128(base + (slot0 + i * 2) * 512), bb = lds128(base + (slot0 + i * 2 + 1) * 512);
-              wa[0] = a.x; wa[1] = a.y; wa[2] = a.z; wa[3] = a.w;
-              wb[0] = bb.x; wb[1] = bb.y; wb[2] = bb.z; wb[3] = bb.w;
-            } else {
-              const uint4 a = lds128(base + (slot0 + i * 2) * 512), bb = lds128(base + (slot0 + i * 2 + 1) * 512);
-              wa[0] = a.x; wa[1] = a.y; wa[2] = a.z; wa[3] = 0u;
-              wb[0] = bb.x; wb[1] = bb.y; wb[2] = bb.z; wb[3] = 0u;
+        for (int i0 = 0; i0 < ROWS_MAX; i0 += RG) {
+          if (i0 < rows) {
+            float d[RG][4];
+            uint32_t wa[RG][4], wb[RG][4];
+#pragma unroll
+            for (int k = 0; k < RG; ++k) {
+              // neighbouring quads walk the group's rows in a rotated order (their rows then sit in different
+              // bank halves); a row past the end of the batch is read from the last row and weighted by zero
+              const int i = min(i0 + ((k + gid) & 3), rows - 1);
+              if (WPT == 4) {
+                const uint4 a = lds128(xa + i * ROWB), bb = lds128(xb + i * ROWB);
+                wa[k][0] = a.x; wa[k][1] = a.y; wa[k][2] = a.z; wa[k][3] = a.w;
+                wb[k][0] = bb.x; wb[k][1] = bb.y; wb[k][2] = bb.z; wb[k][3] = bb.w;
+              } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  wa[k][j] = (j < WPT) ? lds_u32(xa + i * ROWB + j * 4) : 0u;
+                  wb[k][j] = (j < WPT) ? lds_u32(xb + i * ROWB + j * 4) : 0u;
+                }
+              }
+              d[k][0] = d[k][1] = d[k][2] = d[k][3] = 0.f;
             }
 #pragma unroll
             for (int j = 0; j < WPT; ++j) {
-              uint32_t ha[4], hb[4];
-              e2m1x8_to_f16(wa[j], ha);
-              e2m1x8_to_f16(wb[j], hb);
 #pragma unroll
-              for (int t = 0; t < NT; ++t) {
-                mma16816_f16(d0, d1, d2, d3, ha[0], hb[0], ha[1], hb[1], bq[t][2 * j][0], bq[t][2 * j][1]);
-                mma16816_f16(d0, d1, d2, d3, ha[2], hb[2], ha[3], hb[3], bq[t][2 * j + 1][0], bq[t][2 * j + 1][1]);
+              for (int k = 0; k < RG; ++k) {
+                uint32_t ha[4], hb[4];
+                e2m1x8_to_f16(wa[k][j], ha);
+                e2m1x8_to_f16(wb[k][j], hb);
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                  mma16816_f16(d[k][0], d[k][1], d[k][2], d[k][3], ha[0], hb[0], ha[1], hb[1], bq[t][2 * j][0], bq[t][2 * j][1]);
+                  mma16816_f16(d[k][0], d[k][1], d[k][2], d[k][3], ha[2], hb[2], ha[3], hb[3], bq[t][2 * j + 1][0],
+                               bq[t][2 * j + 1][1]);
+                }
               }
             }
-            float sa, sb;
-            if (scale_sz == 4) {
-              sa = lds_f32(sbase + (row0 + i) * 4);
-              sb = lds_f32(sbase + 64 + (row0 + i) * 4);
-            } else {
-              const unsigned char *sp = wsm + st * kScoreStageBytes + kSlots * 512 + (2 * gid) * 64;
-              sa = __half2float(reinterpret_cast<const __half *>(sp)[row0 + i]);
-              sb = __half2float(reinterpret_cast<const __half *>(sp + 64)[row0 + i]);
+#pragma unroll
+            for (int k = 0; k < RG; ++k) {
+              float sa = 0.f, sb = 0.f;
+              if (i0 + ((k + gid) & 3) < rows) {
+                const int ri = row0 + i0 + ((k + gid) & 3);
+                if (scale_sz == 4) {
+                  sa = reinterpret_cast<const float *>(sp)[ri];
+                  sb = reinterpret_cast<const float *>(sp)[r + ri];
+                } else {
+                  sa = __half2float(reinterpret_cast<const __half *>(sp)[ri]);
+                  sb = __half2float(reinterpret_cast<const __half *>(sp)[r + ri]);
+                }
+              }
+              const float d0 = d[k][0] * (sa * m0), d1 = d[k][1] * (sa * m1);
+              const float d2 = d[k][2] * (sb * m0), d3 = d[k][3] * (sb * m1);
+              sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
             }
-            d0 *= sa * m0; d1 *= sa * m1; d2 *= sb * m0; d3 *= sb * m1;
-          } else {
+          }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < ROWS_MAX; ++i) {
+          if (i < rows) {
+            float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
 #pragma unroll
             for (int m = 0; m < MCH; ++m) {
-              const uint4 va = lds128(base + (slot0 + (i * 2) * MCH + m) * 512);
-              const uint4 vb = lds128(base + (slot0 + (i * 2 + 1) * MCH + m) * 512);
+              const uint4 va = lds128(xa + i * ROWB + m * 64), vb = lds128(xb + i * ROWB + m * 64);
               mma16816_bf16(d0, d1, d2, d3, va.x, vb.x, va.y, vb.y, bm[2 * m][0], bm[2 * m][1]);
               mma16816_bf16(d0, d1, d2, d3, va.z, vb.z, va.w, vb.w, bm[2 * m + 1][0], bm[2 * m + 1][1]);
             }
             d0 *= inv_sqrt_d; d1 *= inv_sqrt_d; d2 *= inv_sqrt_d; d3 *= inv_sqrt_d;
+            sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
           }
-          sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
         }
       }
     }
 
+    COBS_ACC(3);
     // ---- end of a chunk: publish t = exp(e - chunk max) per block and the chunk's (max, sum of t) per head ----
     if (cur_b == n_batches - 1) {
       if (pend_u != u && pend_n > 0) {       // moving on to another unit: count the finished one's chunks
@@ -618,10 +723,11 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, int wg, int n_w
       }
       ++pend_n;
     }
-    __syncwarp();
-    cur = nxt; cur_b = nxt_b; st ^= 1;
+    __syncwarp();                           // all lanes are done with stage st before it is refilled
+    COBS_ACC(4);
+    cu = nu; cck = nck; cur_b = nxt_b; st ^= 1;
   }
-  cpa_wait<0>();
+  COBS_ACC_FLUSH(wg);
   if (pend_n > 0) {
     __threadfence();
     __syncwarp();
@@ -663,9 +769,9 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
   // V (transposed): matrices (tokens 0-7, chunk 2np), (8-15, 2np), (0-7, 2np+1), (8-15, 2np+1)
   const int vt = ((lane >> 3) & 1) * 8 + (lane & 7), vc = lane >> 4;
 
-  const long long n_items = (long long)units * n_splits;
-  for (long long item = wg; item < n_items; item += n_wg) {
-    const int u = (int)(item / n_splits), split = (int)(item - (long long)u * n_splits);
+  const int n_items = units * n_splits;
+  for (int item = wg; item < n_items; item += n_wg) {
+    const int u = item / n_splits, split = item - u * n_splits;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
     const int T = p.seq_lens[b_idx];
     const int ws = window_start(T, p.window, L);
@@ -859,19 +965,6 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
   }
 }
 
-#ifdef COBS_TIMING
-// development aid: per-warp phase boundary timestamps (ns), read back by cobs_debug_times
-__device__ unsigned long long g_dbg_times[4][4096];
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define COBS_STAMP(k) do { if (lane == 0 && wg < 4096) g_dbg_times[k][wg] = gtime(); } while (0)
-#else
-#define COBS_STAMP(k) do { } while (0)
-#endif
-
 // ---------------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------------
@@ -881,9 +974,16 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_step_kernel(Params p, int 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = blockIdx.x * kFWarps + warp, n_wg = gridDim.x * kFWarps;
   unsigned char *wsm = fsm + warp * kWarpSmemBytes;
+  __shared__ __align__(8) uint64_t s_bars[kFWarps][2];     // one mbarrier per scoring stage per warp
+  if (lane == 0) {
+    mbar_init((uint32_t)__cvta_generic_to_shared(&s_bars[warp][0]), 1);
+    mbar_init((uint32_t)__cvta_generic_to_shared(&s_bars[warp][1]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
   COBS_STAMP(0);
   if (phases & PH_SCORE) {
-    score_phase<DT, D, WPT, NT>(p, wsm, wg, n_wg, lane);
+    score_phase<DT, D, WPT, NT>(p, wsm, &s_bars[warp][0], wg, n_wg, lane);
     COBS_STAMP(1);
     __syncthreads();                       // the four rings are idle: the selection uses them as one scratch area
     select_phase(p, fsm);
@@ -993,5 +1093,10 @@ cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream) {
 #ifdef COBS_TIMING
 extern "C" int cobs_debug_times(unsigned long long *host_out) {
   return (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_times, sizeof(unsigned long long) * 4 * 4096);
+}
+extern "C" int cobs_debug_acc(unsigned long long *host_out, int clear) {
+  int e = (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_acc, sizeof(unsigned long long) * 8 * 4096);
+  if (clear) { static unsigned long long z[8 * 4096]; cudaMemcpyToSymbol(cobs::g_dbg_acc, z, sizeof(z)); }
+  return e;
 }
 #endif
