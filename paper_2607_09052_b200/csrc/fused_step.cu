@@ -52,6 +52,9 @@ constexpr int kMaxSelectBlocks = 16384;                      // scores + chunk w
 constexpr long long kSpinLimit = 4000000;                    // x ~100 ns: bounded wait on another warp
 
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
+#ifndef COBS_SCORE_RG
+#define COBS_SCORE_RG 4                                      // FP4 factor rows decoded and multiplied together
+#endif
 
 #ifdef COBS_TIMING
 // development aid: per-warp phase boundary timestamps (ns), read back by cobs_debug_times
@@ -428,20 +431,22 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
   // first position at or after (u, ck) that holds work, or u = units when the range is exhausted.
   // Chunk 0 of a unit without summarised blocks counts as work: its warp counts it, so that the
   // selection phase sees the unit as scored.
-  auto seek = [&](int &u, int &ck) {
+  // n_sum of the unit rides along with the position, so that seq_lens is read once per unit.
+  auto unit_blocks = [&](int u) -> int { return min(p.seq_lens[u / p.Hkv] / L, NB); };
+  auto seek = [&](int &u, int &ck, int &n_sum) {
     while (u < units && u * cpu + ck < c_end) {
-      const int n_sum = min(p.seq_lens[u / p.Hkv] / L, NB);
       if (ck * 16 < n_sum || ck == 0) return;
       ++u; ck = 0;                             // rest of this unit has no summaries
+      if (u < units) n_sum = unit_blocks(u);
     }
     u = units;
   };
 
+  COBS_ACC_DECL;
   // ---- bulk copies of (chunk c, batch b) into stage st; completion is counted on the stage's mbarrier ----
   // lanes 0-15 copy the factor rows of block `lane`, lanes 16-31 the mean of block `lane - 16`, lane 0 the scales
-  auto issue = [&](int u, int ck, int b, int st) {
+  auto issue = [&](int u, int ck, int n_sum, int b, int st) {
     if (u >= units) return;
-    const int n_sum = min(p.seq_lens[u / p.Hkv] / L, NB);
     if (ck * 16 >= n_sum) return;
     const int nblk = min(16, NB - ck * 16);
     const size_t rec0 = (size_t)u * NB + ck * 16;
@@ -457,14 +462,24 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
       uint32_t tx = (uint32_t)nblk * (uint32_t)(rows > 0 ? rows * ROWB : 0);
       if (b == 0) tx += (uint32_t)nblk * (D * 2);
       if (scales_bulk) tx += (uint32_t)(16 * r * scale_sz);
-      fence_proxy_async();
       mbar_expect_tx(bar, tx);
+      if (single) {                            // the whole chunk: three contiguous pieces, one lane issues them
+        bulk_g2s(sbase, (const char *)p.mean + rec0 * (size_t)(D * 2), nblk * D * 2, bar);
+        if (rows > 0) bulk_g2s(sbase + xoff, (const char *)p.xi + rec0 * r * (size_t)ROWB, nblk * r * ROWB, bar);
+        if (scales_bulk) bulk_g2s(sbase + soff, (const char *)p.scale + rec0 * (size_t)(r * scale_sz), 16 * r * scale_sz, bar);
+      }
+    }
+    COBS_ACC(5);
+    if (single) {
+      if (FP4 && r > 0 && !scales_bulk) {      // ragged last chunk of the array: plain loads, 4 bytes at a time
+        const char *ssrc = (const char *)p.scale + rec0 * (size_t)(r * scale_sz);
+        for (int w = lane * 4; w < nblk * r * scale_sz; w += 128)
+          *reinterpret_cast<uint32_t *>(wsm + st * kScoreStageBytes + soff + w) = *reinterpret_cast<const uint32_t *>(ssrc + w);
+      }
+      return;
     }
     __syncwarp();
-    if (single) {
-      if (lane == 0) bulk_g2s(sbase, (const char *)p.mean + rec0 * (size_t)(D * 2), nblk * D * 2, bar);
-      if (lane == 1 && rows > 0) bulk_g2s(sbase + xoff, (const char *)p.xi + rec0 * r * (size_t)ROWB, nblk * r * ROWB, bar);
-    } else if (lane < 16) {
+    if (lane < 16) {
       if (lane < nblk && rows > 0)
         bulk_g2s(sbase + xoff + lane * xs, (const char *)p.xi + ((rec0 + lane) * r + row0) * (size_t)ROWB, rows * ROWB, bar);
     } else if (b == 0 && lane - 16 < nblk) {
@@ -481,12 +496,12 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
     }
   };
 
-  int cu = c_begin / cpu, cck = c_begin - cu * cpu;        // current position
-  if (c_begin >= c_end) cu = units; else seek(cu, cck);
+  int cu = c_begin / cpu, cck = c_begin - cu * cpu, cn = 0;   // current position and its unit's block count
+  if (c_begin >= c_end) cu = units; else { cn = unit_blocks(cu); seek(cu, cck, cn); }
   int cur_b = 0, st = 0;
   uint32_t phase_bits = 0;                  // bit st = parity to wait for on stage st
   int pend_u = -1, pend_n = 0;              // chunks finished but not yet counted (counted once per unit run)
-  issue(cu, cck, 0, 0);
+  issue(cu, cck, cn, 0, 0);
   // per-chunk state
   uint32_t bm[KSM][2];
   uint32_t bq[FP4 ? NT : 1][KSQ][2];
@@ -495,22 +510,21 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
   int cur_u = -1;
   bool alive = true;
 
-  COBS_ACC_DECL;
   while (cu < units && alive) {
     COBS_ACC(0);
     // ---- prefetch the next batch of this warp --------------------------------------------------------
-    int nu = cu, nck = cck, nxt_b = cur_b + 1;
+    int nu = cu, nck = cck, nn = cn, nxt_b = cur_b + 1;
     if (nxt_b >= n_batches) {
       nxt_b = 0;
-      if (++nck >= cpu) { ++nu; nck = 0; }
-      seek(nu, nck);
+      if (++nck >= cpu) { ++nu; nck = 0; if (nu < units) nn = unit_blocks(nu); }
+      seek(nu, nck, nn);
     }
-    issue(nu, nck, nxt_b, st ^ 1);
+    COBS_ACC(6);
+    issue(nu, nck, nn, nxt_b, st ^ 1);
     COBS_ACC(1);
 
-    const int u = cu, ck = cck;
+    const int u = cu, ck = cck, n_sum = cn;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
-    const int n_sum = min(p.seq_lens[b_idx] / L, NB);
     const uint32_t sbase = ring + st * kScoreStageBytes;
     if (ck * 16 < n_sum) {
       if (!mbar_wait(bar0 + st * 8, (phase_bits >> st) & 1u)) {     // bounded: the copies never landed
@@ -582,15 +596,16 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
           }
         }
         // ---- first-order term: block means against the raw bf16 query ------------------------------------
-        float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+        float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;   // two chains
         const uint32_t ma = sbase + (2 * gid) * mrow + tig * 16, mb = ma + mrow;
 #pragma unroll
         for (int m = 0; m < MCH; ++m) {
           const uint4 va = lds128(ma + m * 64), vb = lds128(mb + m * 64);
           mma16816_bf16(c0, c1, c2, c3, va.x, vb.x, va.y, vb.y, bm[2 * m][0], bm[2 * m][1]);
-          mma16816_bf16(c0, c1, c2, c3, va.z, vb.z, va.w, vb.w, bm[2 * m + 1][0], bm[2 * m + 1][1]);
+          mma16816_bf16(e0, e1, e2, e3, va.z, vb.z, va.w, vb.w, bm[2 * m + 1][0], bm[2 * m + 1][1]);
         }
-        fA0 = c0 * inv_sqrt_d; fA1 = c1 * inv_sqrt_d; fB0 = c2 * inv_sqrt_d; fB1 = c3 * inv_sqrt_d;
+        fA0 = (c0 + e0) * inv_sqrt_d; fA1 = (c1 + e1) * inv_sqrt_d;
+        fB0 = (c2 + e2) * inv_sqrt_d; fB1 = (c3 + e3) * inv_sqrt_d;
         sA0 = sA1 = sB0 = sB1 = 0.f;
       }
       // ---- curvature term: rows of this batch ----------------------------------------------------------
@@ -599,8 +614,8 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
       const uint32_t xs = (cur_b == 0) ? XS0 : XSN;
       const uint32_t xa = sbase + ((cur_b == 0) ? mean_bytes : 0) + (2 * gid) * xs + tig * (FP4 ? WPT * 4 : 16), xb = xa + xs;
       if (FP4) {
-        // four factor rows at a time: four independent accumulator chains keep the tensor pipe busy
-        constexpr int RG = 4;
+        // RG factor rows at a time: RG independent accumulator chains keep the tensor pipe busy
+        constexpr int RG = COBS_SCORE_RG;
         const unsigned char *sp = wsm + st * kScoreStageBytes + (kScoreStageBytes - scale_bytes) + (2 * gid) * r * scale_sz;
 #pragma unroll
         for (int i0 = 0; i0 < ROWS_MAX; i0 += RG) {
@@ -611,7 +626,7 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
             for (int k = 0; k < RG; ++k) {
               // neighbouring quads walk the group's rows in a rotated order (their rows then sit in different
               // bank halves); a row past the end of the batch is read from the last row and weighted by zero
-              const int i = min(i0 + ((k + gid) & 3), rows - 1);
+              const int i = min(i0 + ((k + gid) & (RG - 1)), rows - 1);
               if (WPT == 4) {
                 const uint4 a = lds128(xa + i * ROWB), bb = lds128(xb + i * ROWB);
                 wa[k][0] = a.x; wa[k][1] = a.y; wa[k][2] = a.z; wa[k][3] = a.w;
@@ -643,8 +658,8 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
 #pragma unroll
             for (int k = 0; k < RG; ++k) {
               float sa = 0.f, sb = 0.f;
-              if (i0 + ((k + gid) & 3) < rows) {
-                const int ri = row0 + i0 + ((k + gid) & 3);
+              if (i0 + ((k + gid) & (RG - 1)) < rows) {
+                const int ri = row0 + i0 + ((k + gid) & (RG - 1));
                 if (scale_sz == 4) {
                   sa = reinterpret_cast<const float *>(sp)[ri];
                   sb = reinterpret_cast<const float *>(sp)[r + ri];
@@ -700,7 +715,7 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
         }
-        const float tA0 = expf(eA0 - mx0), tB0 = expf(eB0 - mx0), tA1 = expf(eA1 - mx1), tB1 = expf(eB1 - mx1);
+        const float tA0 = __expf(eA0 - mx0), tB0 = __expf(eB0 - mx0), tA1 = __expf(eA1 - mx1), tB1 = __expf(eB1 - mx1);
         float *e0 = p.e + ((size_t)u * G + g0) * NB, *e1 = p.e + ((size_t)u * G + g1) * NB;
         if (g0 < G) {
           if (bA < n_sum) __stcg(e0 + bA, tA0);
@@ -725,7 +740,7 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
     }
     __syncwarp();                           // all lanes are done with stage st before it is refilled
     COBS_ACC(4);
-    cu = nu; cck = nck; cur_b = nxt_b; st ^= 1;
+    cu = nu; cck = nck; cn = nn; cur_b = nxt_b; st ^= 1;
   }
   COBS_ACC_FLUSH(wg);
   if (pend_n > 0) {
