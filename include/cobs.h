@@ -198,6 +198,35 @@ int32_t cobs_decode_step_host(const cobs_config *cfg, const void *q_host, const 
                               const cobs_summaries *summ, float *out_host, int32_t *sel_idx_host_or_null,
                               int32_t *sel_cnt_host_or_null, void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * cobs_sparse_decode for callers that cannot provide a workspace.  (The paper has no counterpart: this is
+ * a packaging variant of step (d), same arithmetic and same results as cobs_sparse_decode.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - a decode loop inside a serving
+ * process whose memory pool belongs to another component and is fully handed out, a latency-critical
+ * path where cudaMalloc's device-wide synchronisation is not acceptable, a plug-in that receives only
+ * its input and output tensors.  Such a caller has nowhere to get the split-KV scratch from, so this
+ * variant keeps the scratch (status word, per-unit counters, split partials) in a fixed device array
+ * inside the library: COBS_STATIC_SCRATCH_BYTES per GPU, held from the moment the library is loaded on
+ * that GPU until the process exits.  The call allocates nothing and frees nothing.
+ *
+ * Limits and rules:
+ *   - the configuration's scratch need, 256 + 12 * B * Hkv (rounded up to 256) + B * Hkv * slices * G *
+ *     (D + 2) * 4 bytes, must fit COBS_STATIC_SCRATCH_BYTES, else COBS_ERR_WORKSPACE_TOO_SMALL is
+ *     returned and nothing is launched (the benchmark's 16 x 8 units at G = 4, D = 128 need 2.4 MB);
+ *   - the first call on a device looks up the array's device address (a one-off set-up step); make that
+ *     first call outside any stream capture;
+ *   - all calls on a device share the one array and it keeps the previous call's contents: the call
+ *     itself clears the status word and the counters on `stream` before launching, but two calls that
+ *     may overlap on the GPU (different streams, no dependency) race on it - serialise them;
+ *   - device-side problems are not reported through a status word the caller can read here: an
+ *     out-of-range selection entry or page id is skipped, as in cobs_sparse_decode.
+ * Arguments as for cobs_sparse_decode.
+ */
+#define COBS_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void *q, const cobs_kv *kv, const int32_t *sel_idx,
+                                  const int32_t *sel_cnt, float *out, float *lse_or_null, void *stream);
+
 /* Number of kernels this library has launched in this process so far (host-side counter; the paper
  * has no counterpart: it exists so that a benchmark can state how many launches a timed region held). */
 int64_t cobs_kernel_launches(void);

@@ -23,7 +23,7 @@ SCALE_DTYPES = {"fp32": 0, "fp16": 1}
 EXPORTS = [
     "cobs_status_string", "cobs_padded_sub_dim", "cobs_summary_bytes", "cobs_workspace_bytes", "cobs_reset_status",
     "cobs_read_status", "cobs_build_summaries", "cobs_quantise_xi", "cobs_score_select", "cobs_sparse_decode",
-    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches",
+    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_sparse_decode_static",
 ]
 
 
@@ -184,6 +184,15 @@ def cobs_sparse_decode(cfg: Config, q: torch.Tensor, kv: KV, sel_idx: torch.Tens
     _check(lib().cobs_sparse_decode(C.byref(cfg), _ptr(q), C.byref(kv), _ptr(sel_idx), _ptr(sel_cnt), _ptr(out),
                                     _ptr(lse), _ptr(ws), C.c_size_t(ws.numel()), _stream(stream)),
            "cobs_sparse_decode")
+
+
+def cobs_sparse_decode_static(cfg: Config, q: torch.Tensor, kv: KV, sel_idx: torch.Tensor, sel_cnt: torch.Tensor,
+                              out: torch.Tensor, lse: Optional[torch.Tensor], stream=None):
+    """cobs_sparse_decode without a workspace: the scratch is a fixed device array inside the library, so the
+    call allocates nothing (for callers that are not allowed to allocate device memory).  Raises CobsError(3)
+    when the configuration needs more scratch than the library holds."""
+    _check(lib().cobs_sparse_decode_static(C.byref(cfg), _ptr(q), C.byref(kv), _ptr(sel_idx), _ptr(sel_cnt),
+                                           _ptr(out), _ptr(lse), _stream(stream)), "cobs_sparse_decode_static")
 
 
 def cobs_decode_step(cfg: Config, q: torch.Tensor, kv: KV, summ: SummaryBuffers, out: torch.Tensor,

@@ -156,6 +156,22 @@ static int32_t set_kv(Params &p, const cobs_kv *kv) {
 
 static int32_t cuda_status(cudaError_t e) { return e == cudaSuccess ? COBS_OK : COBS_ERR_CUDA; }
 
+// Validated kernel parameters of an attention-only call whose scratch is not a caller workspace.
+// Fills everything except the scratch pointers (status, counters, partials); reports the attention
+// slices per unit so that the caller can lay its scratch out.
+int32_t prepare_attend_params(const cobs_config *cfg, const void *q, const cobs_kv *kv, const int32_t *sel_idx,
+                              const int32_t *sel_cnt, float *out, float *lse_or_null, Params *p) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if (!q || !aligned16(q) || !sel_idx || !sel_cnt || !out || !aligned16(out)) return COBS_ERR_INVALID_ARG;
+  fill_params(*p, cfg, nullptr);
+  if ((st = set_kv(*p, kv)) != COBS_OK) return st;
+  p->q = static_cast<const __nv_bfloat16 *>(q);
+  p->sel_idx = const_cast<int32_t *>(sel_idx); p->sel_cnt = const_cast<int32_t *>(sel_cnt);
+  p->out = out; p->lse = lse_or_null;
+  return COBS_OK;
+}
+
 }  // namespace cobs
 
 using namespace cobs;

@@ -34,6 +34,8 @@
 // atomicAdd; acquire: volatile read, __threadfence, .cg loads).  Every wait is bounded; on expiry the
 // kernel records COBS_ERR_TIMEOUT, skips the dependent work and returns.  The last CTA to finish puts
 // the counters back to zero, so a workspace needs zeroing only once (cobs_reset_status).
+#include <mutex>
+
 #include "common.cuh"
 
 namespace cobs {
@@ -1103,7 +1105,63 @@ cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream) {
   return cudaErrorInvalidValue;
 }
 
+int32_t prepare_attend_params(const cobs_config *cfg, const void *q, const cobs_kv *kv, const int32_t *sel_idx,
+                              const int32_t *sel_cnt, float *out, float *lse_or_null, Params *p);
+
+// ---------------------------------------------------------------------------------------------------
+// cobs_sparse_decode_static: the attention step with its scratch in device memory the library itself
+// owns, for callers that may not allocate.
+// ---------------------------------------------------------------------------------------------------
+// The scratch lives here, in a file-scope device array.  Every GPU that loads the library holds these
+// bytes until the process exits.  In host code the name below is only a handle: the device address is
+// obtained once per device with cudaGetSymbolAddress and that pointer is what the kernel is given.
+static __device__ __align__(256) unsigned char g_static_scratch[COBS_STATIC_SCRATCH_BYTES];
+
+static void *static_scratch_address(cudaError_t *err) {
+  static void *addr[64] = {nullptr};
+  static std::mutex mu;
+  int dev = 0;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess) return nullptr;
+  if (dev < 0 || dev >= 64) { *err = cudaErrorInvalidDevice; return nullptr; }
+  std::lock_guard<std::mutex> lock(mu);
+  if (!addr[dev]) {
+    void *ptr = nullptr;
+    *err = cudaGetSymbolAddress(&ptr, g_static_scratch);     // the current device's copy of the array
+    if (*err != cudaSuccess) return nullptr;
+    addr[dev] = ptr;
+  }
+  return addr[dev];
+}
+
 }  // namespace cobs
+
+extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void *q, const cobs_kv *kv,
+                                             const int32_t *sel_idx, const int32_t *sel_cnt, float *out,
+                                             float *lse_or_null, void *stream) {
+  using namespace cobs;
+  Params p;
+  int32_t st = prepare_attend_params(cfg, q, kv, sel_idx, sel_cnt, out, lse_or_null, &p);
+  if (st != COBS_OK) return st;
+  // scratch layout: [status word + launch counter: 256 B][3 counters per unit][split partials]
+  const size_t units = (size_t)p.B * p.Hkv;
+  const size_t ctl_bytes = (3 * units * sizeof(int) + 255) / 256 * 256;
+  const size_t partial_bytes = units * p.n_splits * p.G * (size_t)(p.D + 2) * sizeof(float);
+  if (kStatusBytes + ctl_bytes + partial_bytes > (size_t)COBS_STATIC_SCRATCH_BYTES) return COBS_ERR_WORKSPACE_TOO_SMALL;
+  cudaError_t e = cudaSuccess;
+  unsigned char *base = static_cast<unsigned char *>(static_scratch_address(&e));
+  if (!base) return COBS_ERR_CUDA;
+  p.status = reinterpret_cast<int32_t *>(base);
+  p.ctl_done = reinterpret_cast<int *>(base) + 1;
+  p.ctl_score = reinterpret_cast<int *>(base + kStatusBytes);
+  p.ctl_ready = p.ctl_score + units;
+  p.ctl_att = p.ctl_ready + units;
+  p.partial = reinterpret_cast<float *>(base + kStatusBytes + ctl_bytes);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the array keeps whatever the previous call left: the status word and the counters must start at zero
+  if (cudaMemsetAsync(base, 0, kStatusBytes + ctl_bytes, s) != cudaSuccess) return COBS_ERR_CUDA;
+  return launch_fused(p, PH_ATTEND, s) == cudaSuccess ? COBS_OK : COBS_ERR_CUDA;
+}
 
 #ifdef COBS_TIMING
 extern "C" int cobs_debug_times(unsigned long long *host_out) {
