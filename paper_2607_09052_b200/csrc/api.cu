@@ -28,7 +28,7 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 static int padded_sub_dim(int Ds, int /*r*/) { return (Ds + 31) / 32 * 32; }
 
 constexpr int kItemGroups = 256;         // 16-token groups one attention work item may hold
-constexpr int kGridWarps = 148 * 2 * 4;  // warps of the persistent kernel on a B200 (sizing heuristic only)
+constexpr int kGridWarps = 148 * 8;      // streaming warps of the persistent kernel on a B200 (sizing heuristic only)
 
 static int max_items(const cobs_config *c) {
   return c->topk + (c->window + c->block_size - 1) / c->block_size + 1;
@@ -70,7 +70,7 @@ static int32_t validate_config(const cobs_config *c) {
 static int choose_splits(const cobs_config *c) {
   const int units = c->batch * c->n_kv_heads;
   const int groups = max_items(c) * (c->block_size / 16);
-  int s = kGridWarps / units;
+  int s = 2 * kGridWarps / units;          // about two slices per streaming warp: the item queue balances them
   const int need = (groups + kItemGroups - 1) / kItemGroups;
   if (s < need) s = need;
   if (s > groups) s = groups;
@@ -115,6 +115,7 @@ static void fill_params(Params &p, const cobs_config *c, void *workspace) {
     char *base = static_cast<char *>(workspace);
     p.status = reinterpret_cast<int32_t *>(base + w.status);
     p.ctl_done = reinterpret_cast<int *>(base + w.status) + 1;
+    p.ctl_item = reinterpret_cast<int *>(base + w.status) + 2;
     p.ctl_score = reinterpret_cast<int *>(base + w.ctl);
     p.ctl_ready = p.ctl_score + (size_t)p.B * p.Hkv;
     p.ctl_att = p.ctl_ready + (size_t)p.B * p.Hkv;

@@ -33,6 +33,7 @@ struct Params {
   // workspace pieces
   int32_t *status;
   int *ctl_done;              // CTAs of the persistent kernel that have finished
+  int *ctl_item;              // next attention item to hand out
   int *ctl_score;             // [B * Hkv] scored chunks per unit
   int *ctl_ready;             // [B * Hkv] 1 once the unit's selection is written
   int *ctl_att;               // [B * Hkv] attention slices finished per unit

@@ -40,8 +40,10 @@
 
 namespace cobs {
 
-constexpr int kFWarps = 4;
-constexpr int kFThreads = kFWarps * 32;
+constexpr int kFWarps = 8;                                   // streaming warps per CTA (score, then attend)
+constexpr int kSelWarps = 4;                                 // selection team of the CTA
+constexpr int kSelThreads = kSelWarps * 32;
+constexpr int kFThreads = (kFWarps + kSelWarps) * 32;        // one CTA per SM
 constexpr int kScoreStageBytes = 14080;                      // means + factor rows + scales of a 16-block chunk
 constexpr int kAttStages = 3;
 constexpr int kAttStageBytes = 2 * 16 * 128 * 2;             // K + V of one 16-token group, D = 128
@@ -49,11 +51,11 @@ constexpr int kTableEntries = 256;                           // 16-token groups 
 constexpr int kRingBytes = (2 * kScoreStageBytes > kAttStages * kAttStageBytes + kTableEntries * 8)
                                ? 2 * kScoreStageBytes : kAttStages * kAttStageBytes + kTableEntries * 8;
 constexpr int kWarpSmemBytes = kRingBytes;                   // 28160
-constexpr int kFusedSmemBytes = kFWarps * kWarpSmemBytes;    // 112640: two CTAs per SM
-constexpr int kMaxSelectBlocks = 16384;                      // scores + chunk weights of a unit fit the CTA's shared memory
+constexpr int kFusedSmemBytes = kFWarps * kWarpSmemBytes;    // 225280: one CTA per SM
 constexpr long long kSpinLimit = 4000000;                    // x ~100 ns: bounded wait on another warp
 
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
+constexpr int kWaves = 2;                                    // the units are scored in this many waves
 #ifndef COBS_SCORE_RG
 #define COBS_SCORE_RG 4                                      // FP4 factor rows decoded and multiplied together
 #endif
@@ -184,204 +186,210 @@ __device__ __forceinline__ bool wait_flag(const int *flag) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Selection phase.  Unit u is selected by CTA u mod gridDim.x (all four warps together) once all its
-// chunks are scored.  Scoring left, per block, t = exp(e - chunk max) and, per chunk, (max, sum of t):
+// Selection.  Every CTA has a team of four warps that does nothing but select: unit u is selected by the team
+// of CTA u mod gridDim.x as soon as all chunks of the unit are scored, while the CTA's streaming warps carry on
+// scoring later units (the selection is a chain of short dependent steps; it runs in issue slots the streaming
+// warps leave idle).  Scoring left, per block, t = exp(e - chunk max) and, per chunk, (max, sum of t):
 //   lse_g   = log-sum-exp over the chunks of head g
 //   score_b = sum_g t[g][b] * exp(chunk max[g] - lse_g)          (= sum_g exp(e[g][b] - lse_g))
 // then the k largest scores among the candidate blocks, lower index on ties, ascending output.
 // ---------------------------------------------------------------------------------------------------
-__device__ __forceinline__ int cta_exclusive_scan(int v, int *warp_tot, int *total) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int inc = v;
+__device__ __forceinline__ void team_sync() { asm volatile("bar.sync 1, %0;\n" ::"n"(kSelThreads) : "memory"); }
+
+// Selection of one unit with everything in registers: thread t owns chunk t of the unit, i.e. blocks 16 t ...
+// 16 t + 15, whose (max, sum) pairs and t values it reads itself.  Needs n_chunks <= kFThreads and NB % 4 == 0.
+// Called by the 128 threads of the CTA's selection team (tid = index in the team).
+__device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, int tid) {
+  __shared__ float s_m[8][kSelWarps], s_s[8][kSelWarps];
+  __shared__ int s_cnt[2][3][kSelWarps];
+  __shared__ int s_scan[2][kSelWarps];
+  const int warp = tid >> 5, lane = tid & 31;
+  const int G = p.G, NB = p.NB, cpu = (NB + 15) / 16, n_chunks = (n_sum + 15) / 16;
+  const bool mine = tid < n_chunks;
+  // ---- log-sum-exp per head from the chunk pairs -----------------------------------------------------------
+  const float2 *pp = reinterpret_cast<const float2 *>(p.lse_part) + (size_t)u * G * cpu;
+  float2 pr[8];
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  __syncthreads();
-  if (lane == 31) warp_tot[warp] = inc;
-  __syncthreads();
-  int base = 0, tot = 0;
+  for (int g = 0; g < 8; ++g) pr[g] = (g < G && mine) ? __ldcg(pp + (size_t)g * cpu + tid) : make_float2(-INFINITY, 0.f);
 #pragma unroll
-  for (int w = 0; w < kFWarps; ++w) {
-    const int t = warp_tot[w];
-    if (w < warp) base += t;
-    tot += t;
+  for (int g = 0; g < 8; ++g) {
+    if (g < G) {
+      float m = pr[g].x, s = pr[g].y;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+        const float nm = fmaxf(m, om);
+        s = (nm == -INFINITY) ? 0.f : s * __expf(m - nm) + os * __expf(om - nm);
+        m = nm;
+      }
+      if (lane == 0) { s_m[g][warp] = m; s_s[g][warp] = s; }
+    }
   }
-  *total = tot;
-  return base + inc - v;
+  team_sync();
+  float w[8];                                    // exp(chunk max - lse) of this thread's chunk, per head
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    w[g] = 0.f;
+    if (g < G) {
+      float M = -INFINITY;
+#pragma unroll
+      for (int q = 0; q < kSelWarps; ++q) M = fmaxf(M, s_m[g][q]);
+      float S = 0.f;
+#pragma unroll
+      for (int q = 0; q < kSelWarps; ++q) S += (s_m[g][q] == -INFINITY) ? 0.f : s_s[g][q] * expf(s_m[g][q] - M);
+      const float lse = M + logf(S);
+      w[g] = mine ? expf(pr[g].x - lse) : 0.f;
+    }
+  }
+  // ---- scores of this thread's 16 blocks ---------------------------------------------------------------------
+  float sc[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) sc[j] = 0.f;
+  const float *tu = p.e + (size_t)u * G * NB + tid * 16;
+#pragma unroll
+  for (int g0 = 0; g0 < 8; g0 += 4) {
+    if (g0 < G) {
+      float4 x[4][4];
+#pragma unroll
+      for (int g = 0; g < 4; ++g)
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          x[g][q] = (g0 + g < G && mine && tid * 16 + 4 * q < n_sum)
+                        ? __ldcg(reinterpret_cast<const float4 *>(tu + (size_t)(g0 + g) * NB) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        if (g0 + g < G) {
+          const float wg_ = w[g0 + g];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            sc[4 * q + 0] = fmaf(x[g][q].x, wg_, sc[4 * q + 0]); sc[4 * q + 1] = fmaf(x[g][q].y, wg_, sc[4 * q + 1]);
+            sc[4 * q + 2] = fmaf(x[g][q].z, wg_, sc[4 * q + 2]); sc[4 * q + 3] = fmaf(x[g][q].w, wg_, sc[4 * q + 3]);
+          }
+        }
+      }
+    }
+  }
+  uint32_t keys[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const int b = tid * 16 + j;
+    if (b >= n_sum) sc[j] = 0.f;                 // beyond the summarised blocks nothing was written
+    if (p.scores && b < n_sum) p.scores[(size_t)u * NB + b] = sc[j];
+    keys[j] = (b < n_cand) ? __float_as_uint(sc[j]) : 0u;
+  }
+  // ---- top-k ------------------------------------------------------------------------------------------------
+  int32_t *out = p.sel_idx + (size_t)u * p.topk;
+  const int k = min(p.topk, n_cand);
+  if (tid == 0) p.sel_cnt[u] = k;
+  for (int i = k + tid; i < p.topk; i += kSelThreads) out[i] = -1;
+  if (k == n_cand) {
+    for (int i = tid; i < k; i += kSelThreads) out[i] = i;
+    return;
+  }
+  // k-th largest key by bisection on its bits (scores are >= 0, so their bit patterns order like integers):
+  // theta = the largest T with #(key >= T) >= k.  Bit 30 alone, then two bits per round (three trial values,
+  // one CTA barrier per round).
+  int par = 0;
+  auto cta_sums = [&](int c0, int c1, int c2, int &t0, int &t1, int &t2) {
+    c0 = __reduce_add_sync(0xffffffffu, c0); c1 = __reduce_add_sync(0xffffffffu, c1); c2 = __reduce_add_sync(0xffffffffu, c2);
+    if (lane == 0) { s_cnt[par][0][warp] = c0; s_cnt[par][1][warp] = c1; s_cnt[par][2][warp] = c2; }
+    team_sync();
+    t0 = t1 = t2 = 0;
+#pragma unroll
+    for (int q = 0; q < kSelWarps; ++q) { t0 += s_cnt[par][0][q]; t1 += s_cnt[par][1][q]; t2 += s_cnt[par][2][q]; }
+    par ^= 1;
+  };
+  uint32_t theta = 0u;
+  {
+    const uint32_t t = 1u << 30;
+    int c = 0, t0, t1, t2;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) c += (keys[j] >= t);
+    cta_sums(c, 0, 0, t0, t1, t2);
+    if (t0 >= k) theta = t;
+  }
+  for (int bit = 29; bit >= 1; bit -= 2) {
+    const uint32_t ta = theta | (3u << (bit - 1)), tb = theta | (2u << (bit - 1)), tc = theta | (1u << (bit - 1));
+    int ca = 0, cb = 0, cc = 0, na, nb, nc;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) { ca += (keys[j] >= ta); cb += (keys[j] >= tb); cc += (keys[j] >= tc); }
+    cta_sums(ca, cb, cc, na, nb, nc);
+    if (na >= k) theta = ta; else if (nb >= k) theta = tb; else if (nc >= k) theta = tc;
+  }
+  // keep every key above theta and the lowest-index `need_eq` keys equal to it, in index order
+  int n_gt_l = 0, n_eq = 0, d0, d1, d2;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) { n_gt_l += (keys[j] > theta); n_eq += (keys[j] == theta && tid * 16 + j < n_cand); }
+  cta_sums(n_gt_l, 0, 0, d0, d1, d2);
+  const int need_eq = k - d0;
+  auto cta_exclusive = [&](int v, int buf) -> int {
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    if (lane == 31) s_scan[buf][warp] = inc;
+    team_sync();
+    int base = 0;
+#pragma unroll
+    for (int q = 0; q < kSelWarps; ++q) base += (q < warp) ? s_scan[buf][q] : 0;
+    return base + inc - v;
+  };
+  const int eq_base = cta_exclusive(n_eq, 0);
+  int eq_rank = eq_base, n_keep = 0;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (tid * 16 + j < n_cand) {
+      if (keys[j] > theta) ++n_keep;
+      else if (keys[j] == theta) { if (eq_rank < need_eq) ++n_keep; ++eq_rank; }
+    }
+  }
+  int pos = cta_exclusive(n_keep, 1);
+  eq_rank = eq_base;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (tid * 16 + j < n_cand) {
+      bool keep = false;
+      if (keys[j] > theta) keep = true;
+      else if (keys[j] == theta) { keep = eq_rank < need_eq; ++eq_rank; }
+      if (keep && pos < k) out[pos++] = tid * 16 + j;
+    }
+  }
 }
 
-__device__ void select_phase(const Params &p, unsigned char *cta_smem) {
-  __shared__ float s_w[8][kFWarps];          // per head: per-warp (max, sum) while reducing, then the lse
-  __shared__ float s_w2[8][kFWarps];
-  __shared__ float s_lse[8];
-  __shared__ int s_hist[256];
-  __shared__ int s_tot[kFWarps];
-  __shared__ uint32_t s_prefix;
-  __shared__ int s_need, s_ok;
-  float *sc = reinterpret_cast<float *>(cta_smem);             // [NB] scores; the rings are idle in this phase
-  float *cw = sc + p.NB;                                       // [G][chunks] exp(chunk max - lse)
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int units = p.B * p.Hkv, G = p.G, NB = p.NB, cpu = (NB + 15) / 16;
-
+__device__ void select_team(const Params &p, int tid) {
+  __shared__ int s_ok;
+  const int units = p.B * p.Hkv;
   for (int u = blockIdx.x; u < units; u += gridDim.x) {
     const int T = p.seq_lens[u / p.Hkv];
-    const int n_sum = min(T / p.L, NB);
+    const int n_sum = min(T / p.L, p.NB);
     const int n_cand = min(window_start(T, p.window, p.L) / p.L, n_sum);
     const int n_chunks = (n_sum + 15) / 16;
     if (tid == 0) {
       int ok = 0;
       for (long long it = 0; it < kSpinLimit; ++it) {
         if (ld_volatile(p.ctl_score + u) >= max(n_chunks, 1)) { ok = 1; break; }
-        __nanosleep(100);
+        __nanosleep(200);
       }
       if (!ok) report(p.status, COBS_ERR_TIMEOUT);
       s_ok = ok;
     }
-    __syncthreads();
-    if (!s_ok) { __syncthreads(); continue; }                  // never scored: leave the unit unselected
+    team_sync();
+    const int ok = s_ok;
+    team_sync();
+    if (!ok) continue;                         // never scored: leave the unit unselected (its attention times out too)
     __threadfence();
-
-    // ---- chunk pairs -> shared memory (one L2 round trip), lse per head -------------------------------------
-    const float2 *pp = reinterpret_cast<const float2 *>(p.lse_part) + (size_t)u * G * cpu;
-    float2 *pairs = reinterpret_cast<float2 *>(cw + 8 * cpu);   // [G][chunks]
-    for (int i = tid; i < G * n_chunks; i += kFThreads) {
-      const int g = i / n_chunks, c = i - g * n_chunks;
-      pairs[g * cpu + c] = __ldcg(pp + (size_t)g * cpu + c);
-    }
-    __syncthreads();
-    for (int g = 0; g < G; ++g) {
-      float m = -INFINITY, s = 0.f;
-      for (int c = tid; c < n_chunks; c += kFThreads) {
-        const float2 v = pairs[g * cpu + c];
-        const float nm = fmaxf(m, v.x);
-        s = s * expf(m - nm) + v.y * expf(v.x - nm);
-        m = nm;
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
-        const float nm = fmaxf(m, om);
-        s = (nm == -INFINITY) ? 0.f : s * expf(m - nm) + os * expf(om - nm);
-        m = nm;
-      }
-      if (lane == 0) { s_w[g][warp] = m; s_w2[g][warp] = s; }
-    }
-    __syncthreads();
-    if (tid < G) {
-      float M = -INFINITY;
-      for (int w = 0; w < kFWarps; ++w) M = fmaxf(M, s_w[tid][w]);
-      float S = 0.f;
-      for (int w = 0; w < kFWarps; ++w) S += (s_w[tid][w] == -INFINITY) ? 0.f : s_w2[tid][w] * expf(s_w[tid][w] - M);
-      s_lse[tid] = M + logf(S);
-    }
-    __syncthreads();
-    for (int i = tid; i < G * n_chunks; i += kFThreads) {
-      const int g = i / n_chunks, c = i - g * n_chunks;
-      cw[g * cpu + c] = expf(pairs[g * cpu + c].x - s_lse[g]);
-    }
-    __syncthreads();
-    // ---- scores: t values from L2, eight per head per thread in flight ------------------------------------------
-    const float *tu = p.e + (size_t)u * G * NB;
-    for (int b0 = 0; b0 < n_sum; b0 += 8 * kFThreads) {
-      float x[8][8];
-#pragma unroll
-      for (int g = 0; g < 8; ++g)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int b = b0 + tid + kFThreads * j;
-          x[g][j] = (g < G && b < n_sum) ? __ldcg(tu + (size_t)g * NB + b) : 0.f;
-        }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int b = b0 + tid + kFThreads * j;
-        if (b < n_sum) {
-          float sv = 0.f;
-#pragma unroll
-          for (int g = 0; g < 8; ++g)
-            if (g < G) sv = fmaf(x[g][j], cw[g * cpu + (b >> 4)], sv);
-          sc[b] = sv;
-          if (p.scores) p.scores[(size_t)u * NB + b] = sv;
-        }
-      }
-    }
-    __syncthreads();
-
-    // ---- top-k -----------------------------------------------------------------------------------------------
-    int32_t *out = p.sel_idx + (size_t)u * p.topk;
-    const int k = min(p.topk, n_cand);
-    if (tid == 0) p.sel_cnt[u] = k;
-    for (int i = k + tid; i < p.topk; i += kFThreads) out[i] = -1;
-    if (k == n_cand) {
-      for (int i = tid; i < k; i += kFThreads) out[i] = i;
-    } else if (k > 0) {
-      // radix select of the k-th largest key (scores are >= 0: their bit patterns order like integers)
-      if (tid == 0) { s_prefix = 0u; s_need = k; }
-      uint32_t mask = 0u;
-      for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = tid; i < 256; i += kFThreads) s_hist[i] = 0;
-        __syncthreads();
-        const uint32_t prefix = s_prefix;
-        for (int b = tid; b < n_cand; b += kFThreads) {
-          const uint32_t key = __float_as_uint(sc[b]);
-          if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1);
-        }
-        __syncthreads();
-        if (warp == 0) {
-          // lane l owns bins 255 - 8 l ... 248 - 8 l; find the bin where the count from the top reaches `need`
-          const int need = s_need;
-          int mine = 0;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) mine += s_hist[255 - 8 * lane - j];
-          int inc = mine;
-#pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += t;
-          }
-          const int before = inc - mine;
-          if (before < need && inc >= need) {              // exactly one lane
-            int cum = before, bin = 255 - 8 * lane;
-            for (int j = 0; j < 8; ++j, --bin) {
-              if (cum + s_hist[bin] >= need) break;
-              cum += s_hist[bin];
-            }
-            s_need = need - cum;
-            s_prefix = prefix | ((uint32_t)bin << shift);
-          }
-        }
-        mask |= 255u << shift;
-        __syncthreads();
-      }
-      const uint32_t theta = s_prefix;   // key of the k-th largest score
-      const int need_eq = s_need;        // blocks with exactly that key to keep (lowest indices first)
-      // ordered compaction: each thread owns a contiguous index range
-      const int per = (n_cand + kFThreads - 1) / kFThreads;
-      const int lo = min(tid * per, n_cand), hi = min(lo + per, n_cand);
-      int n_eq = 0;
-      for (int b = lo; b < hi; ++b) n_eq += (__float_as_uint(sc[b]) == theta);
-      int total;
-      const int eq_base = cta_exclusive_scan(n_eq, s_tot, &total);
-      int eq_rank = eq_base, n_keep = 0;
-      for (int b = lo; b < hi; ++b) {
-        const uint32_t key = __float_as_uint(sc[b]);
-        if (key > theta) ++n_keep;
-        else if (key == theta) { if (eq_rank < need_eq) ++n_keep; ++eq_rank; }
-      }
-      int pos = cta_exclusive_scan(n_keep, s_tot, &total);
-      eq_rank = eq_base;
-      for (int b = lo; b < hi; ++b) {
-        const uint32_t key = __float_as_uint(sc[b]);
-        bool keep = false;
-        if (key > theta) keep = true;
-        else if (key == theta) { keep = eq_rank < need_eq; ++eq_rank; }
-        if (keep && pos < k) out[pos++] = b;
-      }
-    }
+#ifdef COBS_TIMING
+    if (tid == 0 && u < 1024) g_dbg_acc[0][3000 + u] = gtime();
+#endif
+    select_unit_fast(p, u, n_sum, n_cand, tid);
     __threadfence();
-    __syncthreads();
+    team_sync();
     if (tid == 0) atomicExch(p.ctl_ready + u, 1);
+#ifdef COBS_TIMING
+    if (tid == 0 && u < 1024) g_dbg_acc[1][3000 + u] = gtime();
+#endif
   }
 }
 
@@ -425,23 +433,36 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
   const float inv_sqrt_d = 1.0f / sqrtf((float)D);
   const float ln_l = logf((float)L);
 
-  // This warp's contiguous range of chunks (mostly one unit: its query fragments are built once).
-  // Positions are (unit, chunk-in-unit) pairs advanced incrementally; 32-bit arithmetic throughout.
-  const int total = units * cpu;              // the host refuses configurations where this overflows
-  const int per_warp = (total + n_wg - 1) / n_wg;
-  const int c_begin = min(wg * per_warp, total), c_end = min(c_begin + per_warp, total);
-  // first position at or after (u, ck) that holds work, or u = units when the range is exhausted.
-  // Chunk 0 of a unit without summarised blocks counts as work: its warp counts it, so that the
-  // selection phase sees the unit as scored.
-  // n_sum of the unit rides along with the position, so that seq_lens is read once per unit.
+  // Work order.  The units are scored in kWaves waves (first half, second half); within a wave every streaming
+  // warp takes one contiguous range of the wave's chunks (mostly one unit: its query fragments are built once, and
+  // its finished chunks are counted once).  The selection teams pick up a wave's units while the next wave is being
+  // scored - or, for the last wave, while the first wave's units are being attended.
+  // A position is (unit, chunk-in-unit, blocks of the unit); 32-bit arithmetic throughout.
   auto unit_blocks = [&](int u) -> int { return min(p.seq_lens[u / p.Hkv] / L, NB); };
+  const int n_waves = (units >= 2 * kWaves) ? kWaves : 1;
+  int wave = 0, c_end = 0;
+  auto wave_range = [&](int w, int &cb, int &ce) {          // this warp's chunk range [cb, ce) in wave w
+    const int u0 = (units * w) / n_waves, u1 = (units * (w + 1)) / n_waves;
+    const int tot = (u1 - u0) * cpu, per = (tot + n_wg - 1) / n_wg;   // the host refuses configurations where this overflows
+    cb = u0 * cpu + min(wg * per, tot);
+    ce = u0 * cpu + min(wg * per + per, tot);
+  };
+  // first position at or after (u, ck) that holds work, moving on to the next wave's range when this one is
+  // exhausted; u = units when there is nothing left.  Chunk 0 of a unit without summarised blocks counts as work:
+  // its warp counts it, so that the selection sees the unit as scored.
   auto seek = [&](int &u, int &ck, int &n_sum) {
-    while (u < units && u * cpu + ck < c_end) {
-      if (ck * 16 < n_sum || ck == 0) return;
-      ++u; ck = 0;                             // rest of this unit has no summaries
+    for (;;) {
+      while (u < units && u * cpu + ck < c_end) {
+        if (ck * 16 < n_sum || ck == 0) return;
+        ++u; ck = 0;                           // rest of this unit has no summaries
+        if (u < units) n_sum = unit_blocks(u);
+      }
+      if (++wave >= n_waves) { u = units; return; }
+      int cb;
+      wave_range(wave, cb, c_end);
+      u = cb / cpu; ck = cb - u * cpu;
       if (u < units) n_sum = unit_blocks(u);
     }
-    u = units;
   };
 
   COBS_ACC_DECL;
@@ -498,8 +519,14 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
     }
   };
 
-  int cu = c_begin / cpu, cck = c_begin - cu * cpu, cn = 0;   // current position and its unit's block count
-  if (c_begin >= c_end) cu = units; else { cn = unit_blocks(cu); seek(cu, cck, cn); }
+  int cu, cck, cn = 0;                                        // current position and its unit's block count
+  {
+    int cb;
+    wave_range(0, cb, c_end);
+    cu = cb / cpu; cck = cb - cu * cpu;
+    if (cu < units) cn = unit_blocks(cu);
+    seek(cu, cck, cn);
+  }
   int cur_b = 0, st = 0;
   uint32_t phase_bits = 0;                  // bit st = parity to wait for on stage st
   int pend_u = -1, pend_n = 0;              // chunks finished but not yet counted (counted once per unit run)
@@ -744,7 +771,6 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
     COBS_ACC(4);
     cu = nu; cck = nck; cn = nn; cur_b = nxt_b; st ^= 1;
   }
-  COBS_ACC_FLUSH(wg);
   if (pend_n > 0) {
     __threadfence();
     __syncwarp();
@@ -786,8 +812,15 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
   // V (transposed): matrices (tokens 0-7, chunk 2np), (8-15, 2np), (0-7, 2np+1), (8-15, 2np+1)
   const int vt = ((lane >> 3) & 1) * 8 + (lane & 7), vc = lane >> 4;
 
+  // items are handed out in unit order from a global counter: a warp that arrives late simply takes fewer
   const int n_items = units * n_splits;
-  for (int item = wg; item < n_items; item += n_wg) {
+  COBS_ACC_DECL;
+  for (;;) {
+    COBS_ACC(0);
+    int item = 0;
+    if (lane == 0) item = atomicAdd(p.ctl_item, 1);
+    item = __shfl_sync(0xffffffffu, item, 0);
+    if (item >= n_items) break;
     const int u = item / n_splits, split = item - u * n_splits;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
     const int T = p.seq_lens[b_idx];
@@ -800,6 +833,7 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
     const int g0 = min(split * per, n_groups_u), g1 = min(g0 + per, n_groups_u);
     int n_groups = min(g1 - g0, kTableEntries);
     bool ok = true;
+    COBS_ACC(1);
     if (g0 < n_sel * gpb && n_groups > 0) {
       if (wait_select) {
         ok = wait_flag(p.ctl_ready + u);
@@ -809,6 +843,7 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
         n_sel = min(n_sel, min(__ldcg(p.sel_cnt + u), p.topk));
       }
     }
+    COBS_ACC(2);
     // ---- table of this item's groups -----------------------------------------------------------------
     __syncwarp();
     for (int g = lane; g < n_groups; g += 32) {
@@ -874,6 +909,7 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
       cpa_commit();
     };
 
+    COBS_ACC(3);
     issue(0, 0);
     issue(1, 1);
     int st = 0, st2 = 2;
@@ -934,6 +970,7 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
       st2 = (st2 == kAttStages - 1) ? 0 : st2 + 1;
     }
     cpa_wait<0>();
+    COBS_ACC(4);
 
     // ---- this warp's partial: [G][D + 2] = acc, running max (natural log units), running sum ----------------
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
@@ -950,6 +987,7 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
     }
     __threadfence();
     __syncwarp();
+    COBS_ACC(5);
     int last = 0;
     if (lane == 0) last = (atomicAdd(p.ctl_att + u, 1) + 1 == n_splits);
     last = __shfl_sync(0xffffffffu, last, 0);
@@ -958,19 +996,39 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
       __threadfence();
       const float *pu = p.partial + (size_t)u * n_splits * G * (D + 2);
       for (int g = 0; g < G; ++g) {
-        float M = -INFINITY;
-        for (int s = 0; s < n_splits; ++s) M = fmaxf(M, __ldcg(pu + ((size_t)s * G + g) * (D + 2) + D));
-        float den = 0.f;
+        // the slices' (max, sum) pairs: lane s and s + 32 hold slice s (n_splits <= 64), one round trip
+        float ms[2], ls[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int sidx = lane + 32 * k;
+          const bool have = sidx < n_splits;
+          ms[k] = have ? __ldcg(pu + ((size_t)sidx * G + g) * (D + 2) + D) : -INFINITY;
+          ls[k] = have ? __ldcg(pu + ((size_t)sidx * G + g) * (D + 2) + D + 1) : 0.f;
+        }
+        const float M = warp_max(fmaxf(ms[0], ms[1]));
+        float wv[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) wv[k] = (ms[k] == -INFINITY) ? 0.f : __expf(ms[k] - M);
+        const float den = warp_sum(wv[0] * ls[0] + wv[1] * ls[1]);
         float acc[D / 32];
 #pragma unroll
         for (int k = 0; k < D / 32; ++k) acc[k] = 0.f;
-        for (int s = 0; s < n_splits; ++s) {
-          const float *ps = pu + ((size_t)s * G + g) * (D + 2);
-          const float m = __ldcg(ps + D);
-          const float w = (m == -INFINITY) ? 0.f : __expf(m - M);
-          den = fmaf(w, __ldcg(ps + D + 1), den);
+        // accumulators: four slices' rows in flight at a time
+        for (int s0 = 0; s0 < n_splits; s0 += 4) {
+          float x[4][D / 32], wq[4];
 #pragma unroll
-          for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(w, __ldcg(ps + lane + 32 * k), acc[k]);
+          for (int q = 0; q < 4; ++q) {
+            const int sidx = s0 + q;
+            wq[q] = __shfl_sync(0xffffffffu, (sidx < 32) ? wv[0] : wv[1], sidx & 31);
+            const float *ps = pu + ((size_t)min(sidx, n_splits - 1) * G + g) * (D + 2);
+#pragma unroll
+            for (int k = 0; k < D / 32; ++k) x[q][k] = __ldcg(ps + lane + 32 * k);
+            if (sidx >= n_splits) wq[q] = 0.f;
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+#pragma unroll
+            for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(wq[q], x[q][k], acc[k]);
         }
         const size_t bh = (size_t)b_idx * p.Hq + h * G + g;
 #pragma unroll
@@ -979,36 +1037,39 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
       }
     }
     __syncwarp();
+    COBS_ACC(6);
   }
+  COBS_ACC_FLUSH(wg);
 }
 
 // ---------------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------------
 template <int DT, int D, int WPT, int NT>
-__global__ void __launch_bounds__(kFThreads, 2) fused_step_kernel(Params p, int phases) {
+__global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int phases) {
   extern __shared__ __align__(256) unsigned char fsm[];
+  __shared__ __align__(8) uint64_t s_bars[kFWarps][2];     // one mbarrier per scoring stage per streaming warp
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = blockIdx.x * kFWarps + warp, n_wg = gridDim.x * kFWarps;
-  unsigned char *wsm = fsm + warp * kWarpSmemBytes;
-  __shared__ __align__(8) uint64_t s_bars[kFWarps][2];     // one mbarrier per scoring stage per warp
-  if (lane == 0) {
-    mbar_init((uint32_t)__cvta_generic_to_shared(&s_bars[warp][0]), 1);
-    mbar_init((uint32_t)__cvta_generic_to_shared(&s_bars[warp][1]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-  }
-  __syncwarp();
-  COBS_STAMP(0);
-  if (phases & PH_SCORE) {
-    score_phase<DT, D, WPT, NT>(p, wsm, &s_bars[warp][0], wg, n_wg, lane);
+  if (warp < kFWarps) {
+    // ---- streaming warps: score their chunks, then attend their items -------------------------------------
+    unsigned char *wsm = fsm + warp * kWarpSmemBytes;
+    if (lane == 0) {
+      mbar_init((uint32_t)__cvta_generic_to_shared(&s_bars[warp][0]), 1);
+      mbar_init((uint32_t)__cvta_generic_to_shared(&s_bars[warp][1]), 1);
+      asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncwarp();
+    COBS_STAMP(0);
+    if (phases & PH_SCORE) score_phase<DT, D, WPT, NT>(p, wsm, &s_bars[warp][0], wg, n_wg, lane);
     COBS_STAMP(1);
-    __syncthreads();                       // the four rings are idle: the selection uses them as one scratch area
-    select_phase(p, fsm);
-    __syncthreads();
+    COBS_STAMP(2);
+    if (phases & PH_ATTEND) attend_phase<D>(p, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
+    COBS_STAMP(3);
+  } else if (phases & PH_SCORE) {
+    // ---- selection team ----------------------------------------------------------------------------------------
+    select_team(p, (int)threadIdx.x - kFWarps * 32);
   }
-  COBS_STAMP(2);
-  if (phases & PH_ATTEND) attend_phase<D>(p, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
-  COBS_STAMP(3);
   // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
   __syncthreads();
   __shared__ int is_last;
@@ -1020,7 +1081,7 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_step_kernel(Params p, int 
   if (is_last) {
     const int units = p.B * p.Hkv;
     for (int i = threadIdx.x; i < units; i += kFThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
-    if (threadIdx.x == 0) *p.ctl_done = 0;
+    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; }
   }
 }
 
@@ -1070,7 +1131,7 @@ static cudaError_t launch_fused_t(Params p, int phases, cudaStream_t stream) {
 
 // Whether the persistent kernel covers this configuration's scoring phase.
 bool fused_score_supported(const Params &p) {
-  if (p.NB > kMaxSelectBlocks) return false;
+  if (p.NB > kSelThreads * 16 || p.NB % 4 != 0) return false;   // the selection team holds one chunk per thread
   if (p.summ_dtype == COBS_SUMM_BF16) return p.u_q == nullptr;
   if (p.summ_dtype == COBS_SUMM_FP4_E2M1) {
     if (p.Ds_pad % 32 != 0) return false;
@@ -1153,6 +1214,7 @@ extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void 
   if (!base) return COBS_ERR_CUDA;
   p.status = reinterpret_cast<int32_t *>(base);
   p.ctl_done = reinterpret_cast<int *>(base) + 1;
+  p.ctl_item = reinterpret_cast<int *>(base) + 2;
   p.ctl_score = reinterpret_cast<int *>(base + kStatusBytes);
   p.ctl_ready = p.ctl_score + units;
   p.ctl_att = p.ctl_ready + units;
