@@ -70,7 +70,10 @@ static int32_t validate_config(const cobs_config *c) {
 static int choose_splits(const cobs_config *c) {
   const int units = c->batch * c->n_kv_heads;
   const int groups = max_items(c) * (c->block_size / 16);
-  int s = 2 * kGridWarps / units;          // about two slices per streaming warp: the item queue balances them
+#ifndef COBS_ITEMS_PER_WARP
+#define COBS_ITEMS_PER_WARP 2
+#endif
+  int s = COBS_ITEMS_PER_WARP * kGridWarps / units;   // a few slices per streaming warp: the item queue balances them
   const int need = (groups + kItemGroups - 1) / kItemGroups;
   if (s < need) s = need;
   if (s > groups) s = groups;

@@ -55,7 +55,10 @@ constexpr int kFusedSmemBytes = kFWarps * kWarpSmemBytes;    // 225280: one CTA 
 constexpr long long kSpinLimit = 4000000;                    // x ~100 ns: bounded wait on another warp
 
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
-constexpr int kWaves = 2;                                    // the units are scored in this many waves
+#ifndef COBS_WAVES
+#define COBS_WAVES 4
+#endif
+constexpr int kWaves = COBS_WAVES;                           // the units are scored in this many waves
 #ifndef COBS_SCORE_RG
 #define COBS_SCORE_RG 4                                      // FP4 factor rows decoded and multiplied together
 #endif
