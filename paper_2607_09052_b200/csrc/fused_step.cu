@@ -43,6 +43,7 @@ namespace cobs {
 constexpr int kFWarps = 8;                                   // streaming warps per CTA (score, then attend)
 constexpr int kSelWarps = 4;                                 // selection team of the CTA
 constexpr int kSelThreads = kSelWarps * 32;
+constexpr int kLenCache = 256;                               // sequence lengths cached in shared memory
 constexpr int kFThreads = (kFWarps + kSelWarps) * 32;        // one CTA per SM
 constexpr int kScoreStageBytes = 14080;                      // means + factor rows + scales of a 16-block chunk
 constexpr int kAttStages = 3;
@@ -361,11 +362,11 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
   }
 }
 
-__device__ void select_team(const Params &p, int tid) {
+__device__ void select_team(const Params &p, const int *seq_lens, int tid) {
   __shared__ int s_ok;
   const int units = p.B * p.Hkv;
   for (int u = blockIdx.x; u < units; u += gridDim.x) {
-    const int T = p.seq_lens[u / p.Hkv];
+    const int T = seq_lens[u / p.Hkv];
     const int n_sum = min(T / p.L, p.NB);
     const int n_cand = min(window_start(T, p.window, p.L) / p.L, n_sum);
     const int n_chunks = (n_sum + 15) / 16;
@@ -402,7 +403,8 @@ __device__ void select_team(const Params &p, int tid) {
 // (Ds_pad / 32).  NT: f16 terms of the query (1: full space, 2: fp32 subspace query).
 // ---------------------------------------------------------------------------------------------------
 template <int DT, int D, int WPT, int NT>
-__device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars, int wg, int n_wg, int lane) {
+__device__ void score_phase(const Params &p, const int *seq_lens, unsigned char *wsm, uint64_t *bars, int wg, int n_wg,
+                            int lane) {
   constexpr bool FP4 = (DT == COBS_SUMM_FP4_E2M1);
   constexpr int MCH = D / 32;                 // 16-byte chunks of a bf16 row per thread
   constexpr int KSM = D / 16;                 // k-steps of a bf16 row
@@ -441,7 +443,7 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
   // its finished chunks are counted once).  The selection teams pick up a wave's units while the next wave is being
   // scored - or, for the last wave, while the first wave's units are being attended.
   // A position is (unit, chunk-in-unit, blocks of the unit); 32-bit arithmetic throughout.
-  auto unit_blocks = [&](int u) -> int { return min(p.seq_lens[u / p.Hkv] / L, NB); };
+  auto unit_blocks = [&](int u) -> int { return min(seq_lens[u / p.Hkv] / L, NB); };
   const int n_waves = (units >= 2 * kWaves) ? kWaves : 1;
   int wave = 0, c_end = 0;
   auto wave_range = [&](int w, int &cb, int &ce) {          // this warp's chunk range [cb, ce) in wave w
@@ -785,7 +787,8 @@ __device__ void score_phase(const Params &p, unsigned char *wsm, uint64_t *bars,
 // phase A: attention over (unit, split) items + merge
 // ---------------------------------------------------------------------------------------------------
 template <int D>
-__device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_wg, int lane, bool wait_select) {
+__device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char *wsm, int wg, int n_wg, int lane,
+                             bool wait_select) {
   constexpr int CH = D / 8;                   // 16-byte chunks per row
   constexpr int KS = D / 16;
   constexpr int NTL = D / 8;                  // 8-wide output tiles
@@ -826,7 +829,7 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
     if (item >= n_items) break;
     const int u = item / n_splits, split = item - u * n_splits;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
-    const int T = p.seq_lens[b_idx];
+    const int T = seq_lens[b_idx];
     const int ws = window_start(T, p.window, L);
     const int n_cand = ws / L;
     const int n_win = (T - ws + L - 1) / L;
@@ -835,6 +838,17 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
     const int per = (n_groups_u + n_splits - 1) / n_splits;
     const int g0 = min(split * per, n_groups_u), g1 = min(g0 + per, n_groups_u);
     int n_groups = min(g1 - g0, kTableEntries);
+    // ---- query fragments: rows = heads (zero padded to 16), natural k order.
+    // Loaded first: the loads fly while the warp waits for the unit's selection and builds its group table.
+    uint32_t qa[KS][2];
+    {
+      const uint32_t *qg = reinterpret_cast<const uint32_t *>(p.q + ((size_t)b_idx * p.Hq + h * G + gid) * D);
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        qa[s][0] = (gid < G) ? qg[8 * s + tig] : 0u;
+        qa[s][1] = (gid < G) ? qg[8 * s + 4 + tig] : 0u;
+      }
+    }
     bool ok = true;
     COBS_ACC(1);
     if (g0 < n_sel * gpb && n_groups > 0) {
@@ -873,16 +887,6 @@ __device__ void attend_phase(const Params &p, unsigned char *wsm, int wg, int n_
     }
     __syncwarp();
 
-    // ---- query fragments: rows = heads (zero padded to 16), natural k order -----------------------------
-    uint32_t qa[KS][2];
-    {
-      const uint32_t *qg = reinterpret_cast<const uint32_t *>(p.q + ((size_t)b_idx * p.Hq + h * G + gid) * D);
-#pragma unroll
-      for (int s = 0; s < KS; ++s) {
-        qa[s][0] = (gid < G) ? qg[8 * s + tig] : 0u;
-        qa[s][1] = (gid < G) ? qg[8 * s + 4 + tig] : 0u;
-      }
-    }
     float o[NTL][2];
 #pragma unroll
     for (int n = 0; n < NTL; ++n) o[n][0] = o[n][1] = 0.f;
@@ -1054,6 +1058,14 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
   __shared__ __align__(8) uint64_t s_bars[kFWarps][2];     // one mbarrier per scoring stage per streaming warp
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = blockIdx.x * kFWarps + warp, n_wg = gridDim.x * kFWarps;
+  // sequence lengths are consulted at every change of unit: keep them in shared memory when they fit
+  __shared__ int s_len[kLenCache];
+  const int *seq_lens = p.seq_lens;
+  if (p.B <= kLenCache) {
+    for (int i = threadIdx.x; i < p.B; i += kFThreads) s_len[i] = p.seq_lens[i];
+    __syncthreads();
+    seq_lens = s_len;
+  }
   if (warp < kFWarps) {
     // ---- streaming warps: score their chunks, then attend their items -------------------------------------
     unsigned char *wsm = fsm + warp * kWarpSmemBytes;
@@ -1064,14 +1076,14 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
     }
     __syncwarp();
     COBS_STAMP(0);
-    if (phases & PH_SCORE) score_phase<DT, D, WPT, NT>(p, wsm, &s_bars[warp][0], wg, n_wg, lane);
+    if (phases & PH_SCORE) score_phase<DT, D, WPT, NT>(p, seq_lens, wsm, &s_bars[warp][0], wg, n_wg, lane);
     COBS_STAMP(1);
     COBS_STAMP(2);
-    if (phases & PH_ATTEND) attend_phase<D>(p, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
+    if (phases & PH_ATTEND) attend_phase<D>(p, seq_lens, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
     COBS_STAMP(3);
   } else if (phases & PH_SCORE) {
     // ---- selection team ----------------------------------------------------------------------------------------
-    select_team(p, (int)threadIdx.x - kFWarps * 32);
+    select_team(p, seq_lens, (int)threadIdx.x - kFWarps * 32);
   }
   // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
   __syncthreads();
