@@ -41,7 +41,7 @@ struct Params {
   float *qtilde_out;
   float *e;                   // [B][Hkv][G][NB]
   float *lse_part;            // [B][Hkv][G][ceil(NB / 16)][2] per-chunk (max, sum-exp) of e
-  float *partial;             // [B][Hkv][n_splits][G][D + 2]
+  float *partial;             // [B][Hkv][n_splits] slices of [G][D] accumulators + [G] (max, sum) pairs
   int32_t *sel_idx;           // [B][Hkv][topk]
   int32_t *sel_cnt;           // [B][Hkv]
   float *scores;              // optional [B][Hkv][NB]

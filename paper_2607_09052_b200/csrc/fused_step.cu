@@ -60,6 +60,15 @@ enum { PH_SCORE = 1, PH_ATTEND = 2 };
 #define COBS_WAVES 4
 #endif
 constexpr int kWaves = COBS_WAVES;                           // the units are scored in this many waves
+#ifndef COBS_EVEN_SHARES
+#define COBS_EVEN_SHARES 0                                   // scoring: equal chunk counts per warp instead of ceil-sized ranges
+#endif
+#ifndef COBS_EARLY_FETCH
+#define COBS_EARLY_FETCH 0
+#endif
+#ifndef COBS_DEFER_CLOSE
+#define COBS_DEFER_CLOSE 0
+#endif
 #ifndef COBS_SCORE_RG
 #define COBS_SCORE_RG 4                                      // FP4 factor rows decoded and multiplied together
 #endif
@@ -68,20 +77,29 @@ constexpr int kWaves = COBS_WAVES;                           // the units are sc
 // development aid: per-warp phase boundary timestamps (ns), read back by cobs_debug_times
 __device__ unsigned long long g_dbg_times[4][4096];
 __device__ unsigned long long g_dbg_acc[8][4096];   // per-warp accumulated clock cycles by category
+__device__ unsigned long long g_dbg_trace[32][64];  // event times of every 37th streaming warp
 __device__ __forceinline__ unsigned long long gtime() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
 #define COBS_STAMP(k) do { if (lane == 0 && wg < 4096) g_dbg_times[k][wg] = gtime(); } while (0)
+#define COBS_SEL_STAMP(k) do { if (tid == 0 && u < 1024) g_dbg_acc[k][3000 + u] = gtime(); } while (0)
+#define COBS_TRACE_DECL int trace_n = 0
+#define COBS_TRACE() do { if (lane == 0 && wg % 37 == 0 && trace_n < 64) g_dbg_trace[wg / 37][trace_n++] = gtime(); } while (0)
+#define COBS_TRACE1() do { if (first_chunk) COBS_TRACE(); } while (0)
 #define COBS_ACC_DECL long long acc_t[8] = {0,0,0,0,0,0,0,0}; long long acc_last = clock64()
 #define COBS_ACC(k) do { long long now_ = clock64(); acc_t[k] += now_ - acc_last; acc_last = now_; } while (0)
 #define COBS_ACC_FLUSH(id) do { if ((threadIdx.x & 31) == 0 && (id) < 4096) { for (int k_ = 0; k_ < 8; ++k_) g_dbg_acc[k_][id] += acc_t[k_]; } } while (0)
 #else
 #define COBS_ACC_DECL do { } while (0)
+#define COBS_TRACE_DECL do { } while (0)
+#define COBS_TRACE() do { } while (0)
+#define COBS_TRACE1() do { } while (0)
 #define COBS_ACC(k) do { } while (0)
 #define COBS_ACC_FLUSH(id) do { } while (0)
 #define COBS_STAMP(k) do { } while (0)
+#define COBS_SEL_STAMP(k) do { } while (0)
 #endif
 
 
@@ -229,6 +247,7 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
       if (lane == 0) { s_m[g][warp] = m; s_s[g][warp] = s; }
     }
   }
+  COBS_SEL_STAMP(2);
   team_sync();
   float w[8];                                    // exp(chunk max - lse) of this thread's chunk, per head
 #pragma unroll
@@ -281,6 +300,7 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
     if (p.scores && b < n_sum) p.scores[(size_t)u * NB + b] = sc[j];
     keys[j] = (b < n_cand) ? __float_as_uint(sc[j]) : 0u;
   }
+  COBS_SEL_STAMP(3);
   // ---- top-k ------------------------------------------------------------------------------------------------
   int32_t *out = p.sel_idx + (size_t)u * p.topk;
   const int k = min(p.topk, n_cand);
@@ -320,6 +340,7 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
     cta_sums(ca, cb, cc, na, nb, nc);
     if (na >= k) theta = ta; else if (nb >= k) theta = tb; else if (nc >= k) theta = tc;
   }
+  COBS_SEL_STAMP(4);
   // keep every key above theta and the lowest-index `need_eq` keys equal to it, in index order
   int n_gt_l = 0, n_eq = 0, d0, d1, d2;
 #pragma unroll
@@ -360,6 +381,7 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
       if (keep && pos < k) out[pos++] = tid * 16 + j;
     }
   }
+  COBS_SEL_STAMP(5);
 }
 
 __device__ void select_team(const Params &p, const int *seq_lens, int tid) {
@@ -384,16 +406,12 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid) {
     team_sync();
     if (!ok) continue;                         // never scored: leave the unit unselected (its attention times out too)
     __threadfence();
-#ifdef COBS_TIMING
-    if (tid == 0 && u < 1024) g_dbg_acc[0][3000 + u] = gtime();
-#endif
+    COBS_SEL_STAMP(0);
     select_unit_fast(p, u, n_sum, n_cand, tid);
     __threadfence();
     team_sync();
     if (tid == 0) atomicExch(p.ctl_ready + u, 1);
-#ifdef COBS_TIMING
-    if (tid == 0 && u < 1024) g_dbg_acc[1][3000 + u] = gtime();
-#endif
+    COBS_SEL_STAMP(1);
   }
 }
 
@@ -448,9 +466,18 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   int wave = 0, c_end = 0;
   auto wave_range = [&](int w, int &cb, int &ce) {          // this warp's chunk range [cb, ce) in wave w
     const int u0 = (units * w) / n_waves, u1 = (units * (w + 1)) / n_waves;
-    const int tot = (u1 - u0) * cpu, per = (tot + n_wg - 1) / n_wg;   // the host refuses configurations where this overflows
+    const int tot = (u1 - u0) * cpu;                       // the host refuses configurations where this overflows
+#if COBS_EVEN_SHARES
+    // even shares (they differ by at most one chunk); the warps that get the larger share rotate with the wave
+    int wr = wg + w * (n_wg / n_waves + 1);
+    wr -= (wr / n_wg) * n_wg;
+    cb = u0 * cpu + (int)(((long long)wr * tot) / n_wg);
+    ce = u0 * cpu + (int)(((long long)(wr + 1) * tot) / n_wg);
+#else
+    const int per = (tot + n_wg - 1) / n_wg;
     cb = u0 * cpu + min(wg * per, tot);
     ce = u0 * cpu + min(wg * per + per, tot);
+#endif
   };
   // first position at or after (u, ck) that holds work, moving on to the next wave's range when this one is
   // exhausted; u = units when there is nothing left.  Chunk 0 of a unit without summarised blocks counts as work:
@@ -471,6 +498,8 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   };
 
   COBS_ACC_DECL;
+  COBS_TRACE_DECL;
+  COBS_TRACE();
   // ---- bulk copies of (chunk c, batch b) into stage st; completion is counted on the stage's mbarrier ----
   // lanes 0-15 copy the factor rows of block `lane`, lanes 16-31 the mean of block `lane - 16`, lane 0 the scales
   auto issue = [&](int u, int ck, int n_sum, int b, int st) {
@@ -544,6 +573,9 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   int cur_u = -1;
   bool alive = true;
 
+  bool first_chunk = true;
+  (void)first_chunk;
+  COBS_TRACE();
   while (cu < units && alive) {
     COBS_ACC(0);
     // ---- prefetch the next batch of this warp --------------------------------------------------------
@@ -556,6 +588,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     COBS_ACC(6);
     issue(nu, nck, nn, nxt_b, st ^ 1);
     COBS_ACC(1);
+    COBS_TRACE1();
 
     const int u = cu, ck = cck, n_sum = cn;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
@@ -569,6 +602,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
       phase_bits ^= 1u << st;
       __syncwarp();
       COBS_ACC(2);
+      COBS_TRACE1();
       if (cur_b == 0) {
         if (u != cur_u) {
           cur_u = u;
@@ -629,6 +663,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
             m1 = __shfl_sync(0xffffffffu, mult, (2 * tig + 1) * 4);
           }
         }
+        COBS_TRACE1();
         // ---- first-order term: block means against the raw bf16 query ------------------------------------
         float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;   // two chains
         const uint32_t ma = sbase + (2 * gid) * mrow + tig * 16, mb = ma + mrow;
@@ -727,6 +762,8 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     }
 
     COBS_ACC(3);
+    COBS_TRACE1();
+    first_chunk = false;
     // ---- end of a chunk: publish t = exp(e - chunk max) per block and the chunk's (max, sum of t) per head ----
     if (cur_b == n_batches - 1) {
       if (pend_u != u && pend_n > 0) {       // moving on to another unit: count the finished one's chunks
@@ -734,6 +771,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
         __syncwarp();
         if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
         pend_n = 0;
+        COBS_ACC(7);
       }
       pend_u = u;
       if (ck * 16 < n_sum) {
@@ -774,6 +812,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     }
     __syncwarp();                           // all lanes are done with stage st before it is refilled
     COBS_ACC(4);
+    COBS_TRACE();
     cu = nu; cck = nck; cn = nn; cur_b = nxt_b; st ^= 1;
   }
   if (pend_n > 0) {
@@ -781,6 +820,8 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     __syncwarp();
     if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
   }
+  COBS_ACC(0);
+  COBS_ACC_FLUSH(1200 + wg);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -821,11 +862,108 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
   // items are handed out in unit order from a global counter: a warp that arrives late simply takes fewer
   const int n_items = units * n_splits;
   COBS_ACC_DECL;
+
+  // Closing an item = making its partial visible, counting it, and merging the unit if it was the last slice.
+  // It is put off until the next item's first copies are in flight, so that its round trips cost no bandwidth.
+  auto close_item = [&](int u) {
+    __threadfence();
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) last = (atomicAdd(p.ctl_att + u, 1) + 1 == n_splits);
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+    // ---- merge the unit's partials: o = sum_s e^{m_s - M} acc_s / sum_s e^{m_s - M} l_s -------------------
+    // A slice is [G][D] accumulators followed by [G] (max, sum) pairs.  Few round trips: all pairs at once, then the
+    // accumulators of four slices and up to four heads at a time; the weights sit in the (now idle) copy ring.
+    __threadfence();
+    const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
+    const int SL = G * (D + 2), np = n_splits * G;
+    const float *pu = p.partial + (size_t)u * n_splits * SL;
+    float *sm_w = reinterpret_cast<float *>(wsm);            // [n_splits][G] maxima, then weights
+    float *sm_l = sm_w + kMaxSplits * 8;        // [n_splits][G] sums
+    float *sm_M = sm_l + kMaxSplits * 8;        // [8] maxima, [8] denominators
+    for (int base = 0; base < np; base += 128) {
+      float2 pv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int t = base + lane + 32 * i, sidx = t / G, g = t - sidx * G;
+        pv[i] = (t < np) ? __ldcg(reinterpret_cast<const float2 *>(pu + (size_t)sidx * SL + G * D + 2 * g)) : make_float2(-INFINITY, 0.f);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int t = base + lane + 32 * i;
+        if (t < np) { sm_w[t] = pv[i].x; sm_l[t] = pv[i].y; }
+      }
+    }
+    __syncwarp();
+    {
+      const int g = lane & 7, sub = lane >> 3;
+      float mx = -INFINITY;
+      if (g < G) for (int sidx = sub; sidx < n_splits; sidx += 4) mx = fmaxf(mx, sm_w[sidx * G + g]);
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+      float dn = 0.f;
+      if (g < G) for (int sidx = sub; sidx < n_splits; sidx += 4) {
+        const float m = sm_w[sidx * G + g];
+        const float w = (m == -INFINITY) ? 0.f : __expf(m - mx);
+        dn = fmaf(w, sm_l[sidx * G + g], dn);
+        sm_w[sidx * G + g] = w;
+      }
+      dn += __shfl_xor_sync(0xffffffffu, dn, 8);
+      dn += __shfl_xor_sync(0xffffffffu, dn, 16);
+      if (sub == 0 && g < G) { sm_M[g] = mx; sm_M[8 + g] = dn; }
+    }
+    __syncwarp();
+    constexpr int KV = 4 * D / 64;                           // float2 per lane for four heads
+    for (int gq = 0; gq < G; gq += 4) {
+      const int nv2 = min(4, G - gq) * (D / 2);              // float2 in this group of heads
+      float2 acc[KV];
+#pragma unroll
+      for (int k = 0; k < KV; ++k) acc[k] = make_float2(0.f, 0.f);
+      for (int s0 = 0; s0 < n_splits; s0 += 4) {
+        float2 x[4][KV];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float2 *ps = reinterpret_cast<const float2 *>(pu + (size_t)min(s0 + q, n_splits - 1) * SL + gq * D);
+#pragma unroll
+          for (int k = 0; k < KV; ++k) x[q][k] = (lane + 32 * k < nv2) ? __ldcg(ps + lane + 32 * k) : make_float2(0.f, 0.f);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (s0 + q < n_splits) {
+#pragma unroll
+            for (int k = 0; k < KV; ++k) {
+              const int idx = lane + 32 * k;
+              const float w = (idx < nv2) ? sm_w[(s0 + q) * G + gq + idx / (D / 2)] : 0.f;
+              acc[k].x = fmaf(w, x[q][k].x, acc[k].x);
+              acc[k].y = fmaf(w, x[q][k].y, acc[k].y);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < KV; ++k) {
+        const int idx = lane + 32 * k;
+        if (idx < nv2) {
+          const int head = gq + idx / (D / 2), col = (idx - (idx / (D / 2)) * (D / 2)) * 2;
+          const float den = sm_M[8 + head];
+          const size_t bh = (size_t)b_idx * p.Hq + h * G + head;
+          *reinterpret_cast<float2 *>(p.out + bh * D + col) = make_float2(acc[k].x / den, acc[k].y / den);
+        }
+      }
+      if (p.lse && lane < min(4, G - gq)) {
+        const int head = gq + lane;
+        p.lse[(size_t)b_idx * p.Hq + h * G + head] = sm_M[head] + logf(sm_M[8 + head]);
+      }
+    }
+    __syncwarp();
+  };
+
+  int item = 0, open_u = -1;                     // open_u: unit of the item whose partial is written but not yet closed
+  if (lane == 0) item = atomicAdd(p.ctl_item, 1);
+  item = __shfl_sync(0xffffffffu, item, 0);
   for (;;) {
     COBS_ACC(0);
-    int item = 0;
-    if (lane == 0) item = atomicAdd(p.ctl_item, 1);
-    item = __shfl_sync(0xffffffffu, item, 0);
     if (item >= n_items) break;
     const int u = item / n_splits, split = item - u * n_splits;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
@@ -919,8 +1057,20 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     COBS_ACC(3);
     issue(0, 0);
     issue(1, 1);
+    if (open_u >= 0) close_item(open_u);
+    open_u = -1;
+    COBS_ACC(5);
+    // the next item is drawn two groups before this one ends: its index is there when it is needed
+    int next_item = 0;
+#if COBS_EARLY_FETCH
+    const int fetch_at = n_groups - 2;
+    if (fetch_at < 0 && lane == 0) next_item = atomicAdd(p.ctl_item, 1);
+#else
+    const int fetch_at = -1;
+#endif
     int st = 0, st2 = 2;
     for (int g = 0; g < n_groups; ++g) {
+      if (g == fetch_at && lane == 0) next_item = atomicAdd(p.ctl_item, 1);
       issue(g + 2, st2);
       cpa_wait<2>();
       __syncwarp();
@@ -979,73 +1129,30 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     cpa_wait<0>();
     COBS_ACC(4);
 
-    // ---- this warp's partial: [G][D + 2] = acc, running max (natural log units), running sum ----------------
+    // ---- this warp's partial: [G][D] acc, then [G] (running max in natural log units, running sum) ---------
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
     float *part = p.partial + ((size_t)u * n_splits + split) * G * (D + 2);
     if (gid < G) {
-      float *dst = part + gid * (D + 2);
+      float *dst = part + gid * D;
 #pragma unroll
       for (int n = 0; n < NTL; ++n) __stcg(reinterpret_cast<float2 *>(dst + 8 * n + 2 * tig), make_float2(o[n][0], o[n][1]));
-      if (tig == 0) {
-        __stcg(dst + D, (l_run > 0.f) ? m_run * (sl2 * 0.6931471805599453f) : -INFINITY);
-        __stcg(dst + D + 1, l_run);
-      }
+      if (tig == 0)
+        __stcg(reinterpret_cast<float2 *>(part + G * D + 2 * gid),
+               make_float2((l_run > 0.f) ? m_run * (sl2 * 0.6931471805599453f) : -INFINITY, l_run));
     }
-    __threadfence();
-    __syncwarp();
-    COBS_ACC(5);
-    int last = 0;
-    if (lane == 0) last = (atomicAdd(p.ctl_att + u, 1) + 1 == n_splits);
-    last = __shfl_sync(0xffffffffu, last, 0);
-    if (last) {
-      // ---- merge the unit's partials: o = sum_s e^{m_s - M} acc_s / sum_s e^{m_s - M} l_s -------------------
-      __threadfence();
-      const float *pu = p.partial + (size_t)u * n_splits * G * (D + 2);
-      for (int g = 0; g < G; ++g) {
-        // the slices' (max, sum) pairs: lane s and s + 32 hold slice s (n_splits <= 64), one round trip
-        float ms[2], ls[2];
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          const int sidx = lane + 32 * k;
-          const bool have = sidx < n_splits;
-          ms[k] = have ? __ldcg(pu + ((size_t)sidx * G + g) * (D + 2) + D) : -INFINITY;
-          ls[k] = have ? __ldcg(pu + ((size_t)sidx * G + g) * (D + 2) + D + 1) : 0.f;
-        }
-        const float M = warp_max(fmaxf(ms[0], ms[1]));
-        float wv[2];
-#pragma unroll
-        for (int k = 0; k < 2; ++k) wv[k] = (ms[k] == -INFINITY) ? 0.f : __expf(ms[k] - M);
-        const float den = warp_sum(wv[0] * ls[0] + wv[1] * ls[1]);
-        float acc[D / 32];
-#pragma unroll
-        for (int k = 0; k < D / 32; ++k) acc[k] = 0.f;
-        // accumulators: four slices' rows in flight at a time
-        for (int s0 = 0; s0 < n_splits; s0 += 4) {
-          float x[4][D / 32], wq[4];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int sidx = s0 + q;
-            wq[q] = __shfl_sync(0xffffffffu, (sidx < 32) ? wv[0] : wv[1], sidx & 31);
-            const float *ps = pu + ((size_t)min(sidx, n_splits - 1) * G + g) * (D + 2);
-#pragma unroll
-            for (int k = 0; k < D / 32; ++k) x[q][k] = __ldcg(ps + lane + 32 * k);
-            if (sidx >= n_splits) wq[q] = 0.f;
-          }
-#pragma unroll
-          for (int q = 0; q < 4; ++q)
-#pragma unroll
-            for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(wq[q], x[q][k], acc[k]);
-        }
-        const size_t bh = (size_t)b_idx * p.Hq + h * G + g;
-#pragma unroll
-        for (int k = 0; k < D / 32; ++k) p.out[bh * D + lane + 32 * k] = acc[k] / den;
-        if (p.lse && lane == 0) p.lse[bh] = M + logf(den);
-      }
-    }
-    __syncwarp();
+#if COBS_DEFER_CLOSE
+    open_u = u;
+#else
+    close_item(u);
+#endif
+#if !COBS_EARLY_FETCH
+    if (lane == 0) next_item = atomicAdd(p.ctl_item, 1);
+#endif
+    item = __shfl_sync(0xffffffffu, next_item, 0);
     COBS_ACC(6);
   }
+  if (open_u >= 0) close_item(open_u);
   COBS_ACC_FLUSH(wg);
 }
 
@@ -1243,6 +1350,12 @@ extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void 
 #ifdef COBS_TIMING
 extern "C" int cobs_debug_times(unsigned long long *host_out) {
   return (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_times, sizeof(unsigned long long) * 4 * 4096);
+}
+extern "C" int cobs_debug_trace(unsigned long long *host_out) {
+  int e = (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_trace, sizeof(unsigned long long) * 32 * 64);
+  static unsigned long long z[32 * 64];
+  cudaMemcpyToSymbol(cobs::g_dbg_trace, z, sizeof(z));
+  return e;
 }
 extern "C" int cobs_debug_acc(unsigned long long *host_out, int clear) {
   int e = (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_acc, sizeof(unsigned long long) * 8 * 4096);
