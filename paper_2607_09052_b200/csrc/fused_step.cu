@@ -63,12 +63,6 @@ constexpr int kWaves = COBS_WAVES;                           // the units are sc
 #ifndef COBS_EVEN_SHARES
 #define COBS_EVEN_SHARES 0                                   // scoring: equal chunk counts per warp instead of ceil-sized ranges
 #endif
-#ifndef COBS_EARLY_FETCH
-#define COBS_EARLY_FETCH 0
-#endif
-#ifndef COBS_DEFER_CLOSE
-#define COBS_DEFER_CLOSE 0
-#endif
 #ifndef COBS_SCORE_RG
 #define COBS_SCORE_RG 4                                      // FP4 factor rows decoded and multiplied together
 #endif
@@ -864,7 +858,8 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
   COBS_ACC_DECL;
 
   // Closing an item = making its partial visible, counting it, and merging the unit if it was the last slice.
-  // It is put off until the next item's first copies are in flight, so that its round trips cost no bandwidth.
+  // (Drawing the next item before this one is closed was measured and is slower: a warp that turns out to be the
+  // last of its unit then holds an item back for the length of a merge.)
   auto close_item = [&](int u) {
     __threadfence();
     __syncwarp();
@@ -959,7 +954,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     __syncwarp();
   };
 
-  int item = 0, open_u = -1;                     // open_u: unit of the item whose partial is written but not yet closed
+  int item = 0;
   if (lane == 0) item = atomicAdd(p.ctl_item, 1);
   item = __shfl_sync(0xffffffffu, item, 0);
   for (;;) {
@@ -1057,20 +1052,8 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     COBS_ACC(3);
     issue(0, 0);
     issue(1, 1);
-    if (open_u >= 0) close_item(open_u);
-    open_u = -1;
-    COBS_ACC(5);
-    // the next item is drawn two groups before this one ends: its index is there when it is needed
-    int next_item = 0;
-#if COBS_EARLY_FETCH
-    const int fetch_at = n_groups - 2;
-    if (fetch_at < 0 && lane == 0) next_item = atomicAdd(p.ctl_item, 1);
-#else
-    const int fetch_at = -1;
-#endif
     int st = 0, st2 = 2;
     for (int g = 0; g < n_groups; ++g) {
-      if (g == fetch_at && lane == 0) next_item = atomicAdd(p.ctl_item, 1);
       issue(g + 2, st2);
       cpa_wait<2>();
       __syncwarp();
@@ -1141,18 +1124,13 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
         __stcg(reinterpret_cast<float2 *>(part + G * D + 2 * gid),
                make_float2((l_run > 0.f) ? m_run * (sl2 * 0.6931471805599453f) : -INFINITY, l_run));
     }
-#if COBS_DEFER_CLOSE
-    open_u = u;
-#else
     close_item(u);
-#endif
-#if !COBS_EARLY_FETCH
+    COBS_ACC(5);
+    int next_item = 0;
     if (lane == 0) next_item = atomicAdd(p.ctl_item, 1);
-#endif
     item = __shfl_sync(0xffffffffu, next_item, 0);
     COBS_ACC(6);
   }
-  if (open_u >= 0) close_item(open_u);
   COBS_ACC_FLUSH(wg);
 }
 
@@ -1183,7 +1161,13 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
     }
     __syncwarp();
     COBS_STAMP(0);
+#ifdef COBS_SCORE_WARPS
+    if ((phases & PH_SCORE) && warp < COBS_SCORE_WARPS)
+      score_phase<DT, D, WPT, NT>(p, seq_lens, wsm, &s_bars[warp][0], blockIdx.x * COBS_SCORE_WARPS + warp,
+                                  gridDim.x * COBS_SCORE_WARPS, lane);
+#else
     if (phases & PH_SCORE) score_phase<DT, D, WPT, NT>(p, seq_lens, wsm, &s_bars[warp][0], wg, n_wg, lane);
+#endif
     COBS_STAMP(1);
     COBS_STAMP(2);
     if (phases & PH_ATTEND) attend_phase<D>(p, seq_lens, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
