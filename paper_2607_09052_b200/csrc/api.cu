@@ -93,7 +93,7 @@ static WorkspaceLayout layout_workspace(const cobs_config *c) {
   w.status = off; off += kStatusBytes;
   w.ctl = off; off = align_up(off + 3 * B * Hkv * sizeof(int), 256);     // inside the first kCtlBytes
   w.e = off; off = align_up(off + B * Hq * (size_t)c->max_blocks * sizeof(float), 256);
-  w.lse_part = off; off = align_up(off + B * Hq * (size_t)((c->max_blocks + 15) / 16) * 2 * sizeof(float), 256);
+  w.lse_part = off; off = align_up(off + B * Hq * (size_t)((c->max_blocks + 15) / 16) * 4 * 2 * sizeof(float), 256);   // up to four pairs per chunk
   w.partial = off; off = align_up(off + B * Hkv * (size_t)choose_splits(c) * G * (D + 2) * sizeof(float), 256);
   w.sel_idx = off; off = align_up(off + B * Hkv * (size_t)c->topk * sizeof(int32_t), 256);
   w.sel_cnt = off; off = align_up(off + B * Hkv * sizeof(int32_t), 256);

@@ -34,6 +34,9 @@
 // atomicAdd; acquire: volatile read, __threadfence, .cg loads).  Every wait is bounded; on expiry the
 // kernel records COBS_ERR_TIMEOUT, skips the dependent work and returns.  The last CTA to finish puts
 // the counters back to zero, so a workspace needs zeroing only once (cobs_reset_status).
+#include <cuda.h>
+#include <cuda_fp8.h>
+
 #include <mutex>
 
 #include "common.cuh"
@@ -215,6 +218,8 @@ __device__ __forceinline__ void team_sync() { asm volatile("bar.sync 1, %0;\n" :
 // Selection of one unit with everything in registers: thread t owns chunk t of the unit, i.e. blocks 16 t ...
 // 16 t + 15, whose (max, sum) pairs and t values it reads itself.  Needs n_chunks <= kFThreads and NB % 4 == 0.
 // Called by the 128 threads of the CTA's selection team (tid = index in the team).
+// PPC: (max, sum) pairs per 16-block chunk and head left by the scoring path (1, or 4 = one per four blocks).
+template <int PPC>
 __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, int tid) {
   __shared__ float s_m[8][kSelWarps], s_s[8][kSelWarps];
   __shared__ int s_cnt[2][3][kSelWarps];
@@ -223,10 +228,35 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
   const int G = p.G, NB = p.NB, cpu = (NB + 15) / 16, n_chunks = (n_sum + 15) / 16;
   const bool mine = tid < n_chunks;
   // ---- log-sum-exp per head from the chunk pairs -----------------------------------------------------------
-  const float2 *pp = reinterpret_cast<const float2 *>(p.lse_part) + (size_t)u * G * cpu;
+  const float2 *pp = reinterpret_cast<const float2 *>(p.lse_part) + (size_t)u * G * cpu * PPC;
   float2 pr[8];
+  float msub[8][PPC];                            // PPC > 1: the maxima of the chunk's parts
 #pragma unroll
-  for (int g = 0; g < 8; ++g) pr[g] = (g < G && mine) ? __ldcg(pp + (size_t)g * cpu + tid) : make_float2(-INFINITY, 0.f);
+  for (int g = 0; g < 8; ++g) {
+    pr[g] = make_float2(-INFINITY, 0.f);
+#pragma unroll
+    for (int j = 0; j < PPC; ++j) msub[g][j] = -INFINITY;
+    if (g < G && mine) {
+      if (PPC == 1) {
+        pr[g] = __ldcg(pp + (size_t)g * cpu + tid);
+      } else {
+        float2 part[PPC];
+#pragma unroll
+        for (int j = 0; j < PPC; j += 2) {
+          const float4 v = __ldcg(reinterpret_cast<const float4 *>(pp + ((size_t)g * cpu + tid) * PPC + j));
+          part[j] = make_float2(v.x, v.y);
+          part[j + (PPC > 1 ? 1 : 0)] = make_float2(v.z, v.w);
+        }
+        float m = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < PPC; ++j) { msub[g][j] = part[j].x; m = fmaxf(m, part[j].x); }
+        float sum = 0.f;
+#pragma unroll
+        for (int j = 0; j < PPC; ++j) sum += (part[j].x == -INFINITY) ? 0.f : part[j].y * __expf(part[j].x - m);
+        pr[g] = make_float2(m, sum);
+      }
+    }
+  }
 #pragma unroll
   for (int g = 0; g < 8; ++g) {
     if (g < G) {
@@ -244,9 +274,12 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
   COBS_SEL_STAMP(2);
   team_sync();
   float w[8];                                    // exp(chunk max - lse) of this thread's chunk, per head
+  float wsub[8][PPC];                            // PPC > 1: exp(part max - lse)
 #pragma unroll
   for (int g = 0; g < 8; ++g) {
     w[g] = 0.f;
+#pragma unroll
+    for (int j = 0; j < PPC; ++j) wsub[g][j] = 0.f;
     if (g < G) {
       float M = -INFINITY;
 #pragma unroll
@@ -256,6 +289,10 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
       for (int q = 0; q < kSelWarps; ++q) S += (s_m[g][q] == -INFINITY) ? 0.f : s_s[g][q] * expf(s_m[g][q] - M);
       const float lse = M + logf(S);
       w[g] = mine ? expf(pr[g].x - lse) : 0.f;
+      if (PPC > 1) {
+#pragma unroll
+        for (int j = 0; j < PPC; ++j) wsub[g][j] = (mine && msub[g][j] != -INFINITY) ? expf(msub[g][j] - lse) : 0.f;
+      }
     }
   }
   // ---- scores of this thread's 16 blocks ---------------------------------------------------------------------
@@ -276,9 +313,9 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         if (g0 + g < G) {
-          const float wg_ = w[g0 + g];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
+            const float wg_ = (PPC == 4) ? wsub[g0 + g][PPC == 4 ? q : 0] : w[g0 + g];
             sc[4 * q + 0] = fmaf(x[g][q].x, wg_, sc[4 * q + 0]); sc[4 * q + 1] = fmaf(x[g][q].y, wg_, sc[4 * q + 1]);
             sc[4 * q + 2] = fmaf(x[g][q].z, wg_, sc[4 * q + 2]); sc[4 * q + 3] = fmaf(x[g][q].w, wg_, sc[4 * q + 3]);
           }
@@ -378,7 +415,10 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
   COBS_SEL_STAMP(5);
 }
 
-__device__ void select_team(const Params &p, const int *seq_lens, int tid) {
+// count_mult: how often the scoring path counts a chunk on its unit; empty_need: the count a unit without
+// summarised blocks reaches.
+template <int PPC>
+__device__ void select_team(const Params &p, const int *seq_lens, int tid, int count_mult, int empty_need) {
   __shared__ int s_ok;
   const int units = p.B * p.Hkv;
   for (int u = blockIdx.x; u < units; u += gridDim.x) {
@@ -389,7 +429,7 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid) {
     if (tid == 0) {
       int ok = 0;
       for (long long it = 0; it < kSpinLimit; ++it) {
-        if (ld_volatile(p.ctl_score + u) >= max(n_chunks, 1)) { ok = 1; break; }
+        if (ld_volatile(p.ctl_score + u) >= (n_chunks > 0 ? n_chunks * count_mult : empty_need)) { ok = 1; break; }
         __nanosleep(200);
       }
       if (!ok) report(p.status, COBS_ERR_TIMEOUT);
@@ -401,7 +441,7 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid) {
     if (!ok) continue;                         // never scored: leave the unit unselected (its attention times out too)
     __threadfence();
     COBS_SEL_STAMP(0);
-    select_unit_fast(p, u, n_sum, n_cand, tid);
+    select_unit_fast<PPC>(p, u, n_sum, n_cand, tid);
     __threadfence();
     team_sync();
     if (tid == 0) atomicExch(p.ctl_ready + u, 1);
@@ -1135,6 +1175,362 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
 }
 
 // ---------------------------------------------------------------------------------------------------
+// phase S on the 5th-generation tensor cores (tcgen05), for the main configuration: packed E2M1 factors in
+// the full key space, D = 128, r = 8.
+//
+// A 16-block chunk is ONE matrix product: the chunk's 16 x 8 = 128 factor rows (M = 128, K = 128) against the G
+// query heads.  The factor rows are fetched by a tiled TMA copy whose element type makes the copy engine unpack
+// the 4-bit codes into the 8-bit containers `tcgen05.mma.kind::f8f6f4` reads (128-byte swizzled rows in shared
+// memory), so no thread ever touches a code.  The query cannot be FP4: it enters as TWO E4M3 terms per head
+// (high part + remainder of the bf16 query scaled by a power of two: together exact for every element within
+// 2^-10 of the head's largest), columns h and 8 + h of a 16-column operand.  The accumulator (128 lanes x 16
+// fp32 columns) lives in tensor memory, four buffers deep.
+//
+// Roles inside the CTA (one CTA per SM): warp 12 = producer (TMA / bulk copies of factor rows, means, scales; builds
+// the query operand when the unit changes), warp 13 = MMA issuer (one thread), warps 0-3 and 4-7 = two epilogue
+// sets taking alternate chunks (warp w reads the TMEM lanes 32 (w mod 4) ..., i.e. blocks 4 (w mod 4) ... of the
+// chunk), warps 8-11 = the selection team as before.  All hand-offs are mbarriers with bounded waits.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kUStages = 9;                                   // chunks in flight per CTA
+constexpr int kUStageBytes = 21504;                           // 16384 unpacked factor rows + 4096 means + 512 scales, padded to 1 KiB
+constexpr int kUMeanOff = 16384, kUScaleOff = 20480;
+constexpr int kUTiles = 4;                                    // query operands (one per unit) kept at a time
+constexpr int kUTileBytes = 5120;                             // 2048 operand tile + 2048 bf16 query rows + head factors
+constexpr int kUTileQOff = 2048, kUTileFOff = 4096;
+constexpr int kUTilesOff = kUStages * kUStageBytes;           // 193536
+constexpr int kUSmemBytes = kFusedSmemBytes + 1024;           // + slack to align the base to 1 KiB
+static_assert(kUTilesOff + kUTiles * kUTileBytes <= kFusedSmemBytes, "tcgen05 scoring layout exceeds the CTA's shared memory");
+constexpr int kUThreads = (kFWarps + kSelWarps + 2) * 32;     // + producer warp + MMA warp
+constexpr int kUAccCols = 16, kUAccBufs = 4;                  // tensor memory: 64 columns
+constexpr int kUWaitLimit = 2000000;                          // bounded mbarrier waits (try_wait iterations)
+// mbarrier indices
+constexpr int kBFull = 0, kBEmpty = kBFull + kUStages, kBTFull = kBEmpty + kUStages, kBTEmpty = kBTFull + kUAccBufs,
+              kBQFull = kBTEmpty + kUAccBufs, kBCount = kBQFull + kUTiles;
+
+__device__ __forceinline__ bool mbar_wait_lim(uint32_t bar, uint32_t parity) {
+  for (int it = 0; it < kUWaitLimit; ++it) {
+    uint32_t done;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+// K-major operand, 128-byte swizzled rows, 8-row groups 1024 bytes apart (shared-memory matrix descriptor)
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) |
+         (uint64_t(2) << 61);
+}
+// D fp32, A = E2M1, B = E4M3, both K-major, M = 128, N = 16
+constexpr uint32_t kUInstrDesc = (1u << 4) | (5u << 7) | (0u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+
+// The CTA's chunk list: wave by wave, a contiguous range of each wave's chunks, chunks past a unit's summarised
+// blocks left out.  Every role walks the same list with the same sequence numbers.
+struct UmmaIter {
+  int wave, left, u, ck, n_sum, units, cpu, n_waves;
+  __device__ void load_unit(const Params &p, const int *seq_lens) {
+    n_sum = (u < units) ? min(seq_lens[u / p.Hkv] / p.L, p.NB) : 0;
+  }
+  __device__ void open_wave(const Params &p, const int *seq_lens, int w) {
+    wave = w;
+    const int u0 = (units * w) / n_waves, u1 = (units * (w + 1)) / n_waves;
+    const int tot = (u1 - u0) * cpu, per = (tot + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int c = min((int)blockIdx.x * per, tot), c_end = min((int)blockIdx.x * per + per, tot);
+    left = c_end - c;
+    u = u0 + c / cpu;
+    ck = c - (c / cpu) * cpu;
+    load_unit(p, seq_lens);
+  }
+  __device__ void init(const Params &p, const int *seq_lens) {
+    units = p.B * p.Hkv; cpu = (p.NB + 15) / 16;
+    n_waves = (units >= 2 * kWaves) ? kWaves : 1;
+    open_wave(p, seq_lens, 0);
+  }
+  // the next chunk (unit, chunk in unit, summarised blocks of the unit); false at the end of the list
+  __device__ bool next(const Params &p, const int *seq_lens, int &ou, int &ock, int &on_sum) {
+    for (;;) {
+      if (left <= 0) {
+        if (wave + 1 >= n_waves) return false;
+        open_wave(p, seq_lens, wave + 1);
+        continue;
+      }
+      if (ck * 16 < n_sum) {
+        ou = u; ock = ck; on_sum = n_sum;
+        --left;
+        if (++ck == cpu) { ++u; ck = 0; load_unit(p, seq_lens); }
+        return true;
+      }
+      left -= cpu - ck;                          // the rest of this unit has no summaries
+      ++u; ck = 0;
+      load_unit(p, seq_lens);
+    }
+  }
+};
+
+__device__ __forceinline__ void umma_abort(const Params &p, volatile int *abort_flag, int lane) {
+  if (lane == 0) { report(p.status, COBS_ERR_TIMEOUT); *abort_flag = 1; }
+}
+
+// Producer warp: keeps kUStages chunks in flight and builds the query operand of every unit the CTA meets.
+__device__ void umma_producer(const Params &p, const int *seq_lens, unsigned char *fsm, uint32_t bars, const CUtensorMap *tmap,
+                              int lane, volatile int *abort_flag) {
+  UmmaIter it;
+  it.init(p, seq_lens);
+  const int G = p.G, NB = p.NB;
+  const int scale_sz = (p.scale_dtype == COBS_SCALE_FP16) ? 2 : 4;
+  const uint32_t scale_bytes = 16 * 8 * scale_sz;
+  const uint32_t sm = (uint32_t)__cvta_generic_to_shared(fsm);
+  const float inv_sqrt_d = 1.0f / sqrtf(128.0f);
+  int n = 0, cur_u = -1, tile_seq = -1, u = 0, ck = 0, n_sum = 0;
+  COBS_ACC_DECL;
+  while (it.next(p, seq_lens, u, ck, n_sum)) {
+    if (*abort_flag) break;
+    const int slot = n % kUStages;
+    COBS_ACC(0);
+    if (n >= kUStages && !mbar_wait_lim(bars + (kBEmpty + slot) * 8, ((n / kUStages) - 1) & 1)) { umma_abort(p, abort_flag, lane); break; }
+    COBS_ACC(1);
+    if (u != cur_u) {
+      // ---- query operand of unit u: rows h (high E4M3 term) and 8 + h (remainder), 128-byte swizzled ----------
+      cur_u = u;
+      ++tile_seq;
+      unsigned char *tile = fsm + kUTilesOff + (tile_seq & (kUTiles - 1)) * kUTileBytes;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) reinterpret_cast<uint4 *>(tile)[lane * 4 + j] = make_uint4(0, 0, 0, 0);
+      __syncwarp();
+      const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
+      for (int g = 0; g < G; ++g) {
+        const __nv_bfloat16 *qrow = p.q + ((size_t)b_idx * p.Hq + h * G + g) * 128;
+        const uint2 raw = *reinterpret_cast<const uint2 *>(qrow + 4 * lane);
+        const float x0 = bf16_lo(raw.x), x1 = bf16_hi(raw.x), x2 = bf16_lo(raw.y), x3 = bf16_hi(raw.y);
+        const float mx = warp_max(fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3))));
+        int ex = 0;
+        if (mx > 0.f) frexpf(mx, &ex);
+        const float sc = ldexpf(1.0f, 8 - ex);               // largest |q| of the head lands in [128, 256)
+        const float y0 = x0 * sc, y1 = x1 * sc, y2 = x2 * sc, y3 = x3 * sc;
+        const __nv_fp8x2_storage_t h01 = __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);
+        const __nv_fp8x2_storage_t h23 = __nv_cvt_float2_to_fp8x2(make_float2(y2, y3), __NV_SATFINITE, __NV_E4M3);
+        const __half2_raw b01 = __nv_cvt_fp8x2_to_halfraw2(h01, __NV_E4M3), b23 = __nv_cvt_fp8x2_to_halfraw2(h23, __NV_E4M3);
+        const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&b01));
+        const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&b23));
+        const __nv_fp8x2_storage_t l01 = __nv_cvt_float2_to_fp8x2(make_float2(y0 - f01.x, y1 - f01.y), __NV_SATFINITE, __NV_E4M3);
+        const __nv_fp8x2_storage_t l23 = __nv_cvt_float2_to_fp8x2(make_float2(y2 - f23.x, y3 - f23.y), __NV_SATFINITE, __NV_E4M3);
+        const uint32_t hi4 = (uint32_t)h01 | ((uint32_t)h23 << 16), lo4 = (uint32_t)l01 | ((uint32_t)l23 << 16);
+        const int kb = 4 * lane;                            // byte (= element) position in the row
+        const int nh = g, nl = 8 + g;
+        *reinterpret_cast<uint32_t *>(tile + (nh >> 3) * 1024 + (nh & 7) * 128 + (((kb >> 4) ^ (nh & 7)) << 4) + (kb & 15)) = hi4;
+        *reinterpret_cast<uint32_t *>(tile + (nl >> 3) * 1024 + (nl & 7) * 128 + (((kb >> 4) ^ (nl & 7)) << 4) + (kb & 15)) = lo4;
+        *reinterpret_cast<uint2 *>(tile + kUTileQOff + g * 256 + lane * 8) = raw;
+        if (lane == 0) reinterpret_cast<float *>(tile + kUTileFOff)[g] = ldexpf(1.0f, ex - 8) * inv_sqrt_d;
+      }
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + (kBQFull + (tile_seq & (kUTiles - 1))) * 8);
+    }
+    {
+      // lane 0: the factor rows (tensor copy); lanes 1 and 2: the means and the scales (one bulk-copy instruction)
+      const uint32_t st = sm + slot * kUStageBytes, bar = bars + (kBFull + slot) * 8;
+      const uint32_t rec0 = (uint32_t)(u * NB + ck * 16);        // < 2^28 (checked on the host)
+      if (lane == 0) {
+        mbar_expect_tx(bar, 8192u + 4096u + scale_bytes);
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+                     ::"r"(st), "l"(tmap), "r"(0), "r"((int)(rec0 * 8u)), "r"(bar) : "memory");
+      } else if (lane < 3) {
+        const bool is_mean = lane == 1;
+        const char *src = is_mean ? (const char *)p.mean + (size_t)rec0 * 256 : (const char *)p.scale + (size_t)rec0 * (8 * scale_sz);
+        bulk_g2s(st + (is_mean ? kUMeanOff : kUScaleOff), src, is_mean ? 4096u : scale_bytes, bar);
+      }
+    }
+    COBS_ACC(2);
+    ++n;
+  }
+  COBS_ACC_FLUSH((int)blockIdx.x);
+}
+
+// MMA issuer (one thread): one 128 x 16 x 128 product per chunk into the next accumulator buffer.
+__device__ void umma_issuer(const Params &p, const int *seq_lens, unsigned char *fsm, uint32_t bars, uint32_t tmem,
+                            volatile int *abort_flag) {
+  UmmaIter it;
+  it.init(p, seq_lens);
+  const uint64_t desc0 = umma_desc((uint32_t)__cvta_generic_to_shared(fsm));   // the whole region lies below 2^18
+  int n = 0, cur_u = -1, tile_seq = -1, u = 0, ck = 0, n_sum = 0;
+  COBS_ACC_DECL;
+  while (it.next(p, seq_lens, u, ck, n_sum)) {
+    if (*abort_flag) break;
+    const int slot = n % kUStages, acc = n % kUAccBufs;
+    bool ok = true;
+    COBS_ACC(0);
+    if (u != cur_u) {
+      cur_u = u;
+      ++tile_seq;
+      ok = mbar_wait_lim(bars + (kBQFull + (tile_seq & (kUTiles - 1))) * 8, (tile_seq / kUTiles) & 1);
+    }
+    COBS_ACC(1);
+    ok = ok && mbar_wait_lim(bars + (kBFull + slot) * 8, (n / kUStages) & 1);
+    COBS_ACC(2);
+    if (ok && n >= kUAccBufs) ok = mbar_wait_lim(bars + (kBTEmpty + acc) * 8, ((n / kUAccBufs) - 1) & 1);
+    COBS_ACC(3);
+    if (!ok) { umma_abort(p, abort_flag, 0); break; }
+    tc_fence_after();
+    const uint64_t da0 = desc0 + (uint64_t)((slot * kUStageBytes) >> 4);
+    const uint64_t db0 = desc0 + (uint64_t)((kUTilesOff + (tile_seq & (kUTiles - 1)) * kUTileBytes) >> 4);
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      const uint64_t da = da0 + 2 * ks, db = db0 + 2 * ks;     // 32 bytes along K per step
+      const uint32_t accum = ks > 0;
+      asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}\n"
+                   ::"r"(tmem + acc * kUAccCols), "l"(da), "l"(db), "r"(kUInstrDesc), "r"(accum) : "memory");
+    }
+    tc_commit(bars + (kBEmpty + slot) * 8);
+    tc_commit(bars + (kBTFull + acc) * 8);
+    COBS_ACC(4);
+    ++n;
+  }
+  COBS_ACC_FLUSH(200 + (int)blockIdx.x);
+}
+
+// Epilogue warp (streaming warps 0-7; set = warp / 4 takes the chunks of its parity, warp mod 4 = TMEM lane quarter):
+// lane (bl, i) = (lane / 8, lane % 8) holds accumulator row (block 4 q + bl of the chunk, factor i).
+// Leaves per block t = exp(e - chunk max) and per chunk the (max, sum) pairs, like the mma.sync path; each warp
+// counts the chunk on the unit once, so a unit is complete at 4 x its chunks.
+__device__ void umma_epilogue(const Params &p, const int *seq_lens, unsigned char *fsm, uint32_t bars, uint32_t tmem, int warp,
+                              int lane, volatile int *abort_flag) {
+  const int set = warp >> 2, q = warp & 3;
+  const int gid = lane >> 2, tig = lane & 3;      // mma.sync fragment coordinates (mean term)
+  const int bl = lane >> 3, i = lane & 7;
+  const int G = p.G, NB = p.NB, cpu = (NB + 15) / 16;
+  const bool scale_f16 = p.scale_dtype == COBS_SCALE_FP16;
+  const float inv_sqrt_d = 1.0f / sqrtf(128.0f), ln_l = logf((float)p.L);
+  UmmaIter it;
+  it.init(p, seq_lens);
+  int n = 0, j = 0, cur_u = -1, tile_seq = -1, my_u = -1, pend_u = -1, pend_n = 0, u = 0, ck = 0, n_sum = 0;
+  uint32_t bm[8][2];
+  float fac = 0.f;
+#pragma unroll
+  for (int m = 0; m < 8; ++m) bm[m][0] = bm[m][1] = 0u;
+  auto flush = [&]() {
+    if (pend_n > 0) {
+      __threadfence();
+      __syncwarp();
+      if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
+      pend_n = 0;
+    }
+  };
+  COBS_ACC_DECL;
+  while (it.next(p, seq_lens, u, ck, n_sum)) {
+    if (u != cur_u) { cur_u = u; ++tile_seq; }
+    if ((n & 1) != set) { ++n; continue; }
+    if (*abort_flag) break;
+    COBS_ACC(0);
+    const int slot = n % kUStages, acc = n % kUAccBufs;
+    const unsigned char *tile = fsm + kUTilesOff + (tile_seq & (kUTiles - 1)) * kUTileBytes;
+    if (u != my_u) {
+      if (!mbar_wait_lim(bars + (kBQFull + (tile_seq & (kUTiles - 1))) * 8, (tile_seq / kUTiles) & 1)) { umma_abort(p, abort_flag, lane); break; }
+      my_u = u;
+      const uint32_t qs = (uint32_t)__cvta_generic_to_shared(tile + kUTileQOff);
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (gid < G) v = lds128(qs + gid * 256 + (tig + 4 * m) * 16);
+        bm[2 * m][0] = v.x; bm[2 * m][1] = v.y; bm[2 * m + 1][0] = v.z; bm[2 * m + 1][1] = v.w;
+      }
+      fac = (i < G) ? reinterpret_cast<const float *>(tile + kUTileFOff)[i] : 0.f;
+    }
+    COBS_ACC(1);
+    if (!mbar_wait_lim(bars + (kBFull + slot) * 8, (n / kUStages) & 1)) { umma_abort(p, abort_flag, lane); break; }
+    COBS_ACC(2);
+    const unsigned char *stg = fsm + slot * kUStageBytes;
+    // ---- first-order term of blocks 4 q .. 4 q + 3 (rows 0-3 of an m16n8k16 tile; columns = heads) ------------
+    float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;
+    {
+      const uint32_t ma = (uint32_t)__cvta_generic_to_shared(stg + kUMeanOff) + (4 * q + (gid & 3)) * 256 + tig * 16;
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        uint4 va = lds128(ma + m * 64);
+        if (gid >= 4) va = make_uint4(0, 0, 0, 0);
+        mma16816_bf16(c0, c1, c2, c3, va.x, 0u, va.y, 0u, bm[2 * m][0], bm[2 * m][1]);
+        mma16816_bf16(e0, e1, e2, e3, va.z, 0u, va.w, 0u, bm[2 * m + 1][0], bm[2 * m + 1][1]);
+      }
+    }
+    const float f0 = (c0 + e0) * inv_sqrt_d, f1 = (c1 + e1) * inv_sqrt_d;     // lane (gid < 4, tig): block 4q+gid, heads 2tig, 2tig+1
+    const int srow = (4 * q + bl) * 8 + i;
+    const float sc = scale_f16 ? __half2float(reinterpret_cast<const __half *>(stg + kUScaleOff)[srow])
+                               : reinterpret_cast<const float *>(stg + kUScaleOff)[srow];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bars + (kBEmpty + slot) * 8);      // this warp is done with the stage
+    // ---- the chunk's product from tensor memory ---------------------------------------------------------------
+    COBS_ACC(3);
+    if (!mbar_wait_lim(bars + (kBTFull + acc) * 8, (n / kUAccBufs) & 1)) { umma_abort(p, abort_flag, lane); break; }
+    COBS_ACC(4);
+    tc_fence_after();
+    uint32_t r[16];
+    {
+      const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + acc * kUAccCols;
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+                   : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                     "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                   : "r"(taddr));
+      asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bars + (kBTEmpty + acc) * 8);
+    float v[8];
+#pragma unroll
+    for (int h = 0; h < 8; ++h) {
+      const float x = (__uint_as_float(r[h]) + __uint_as_float(r[8 + h])) * sc;
+      v[h] = x * x;
+    }
+    // sum over the 8 factors of a block, transposing as it goes: lane i ends with head i
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float keep = (i & 4) ? v[k + 4] : v[k], send = (i & 4) ? v[k] : v[k + 4];
+      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const float keep = (i & 2) ? v[k + 2] : v[k], send = (i & 2) ? v[k] : v[k + 2];
+      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    float ssum;
+    {
+      const float keep = (i & 1) ? v[1] : v[0], send = (i & 1) ? v[0] : v[1];
+      ssum = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+    }
+    const int src = bl * 4 + (i >> 1);
+    const float fa = __shfl_sync(0xffffffffu, f0, src), fb = __shfl_sync(0xffffffffu, f1, src);
+    const int blk = ck * 16 + 4 * q + bl;
+    const bool live = (i < G) && (blk < n_sum);
+    const float e = live ? ln_l + ((i & 1) ? fb : fa) + 0.5f * (fac * fac) * ssum : -INFINITY;
+    // ---- max and sum per head over the warp's four blocks: one pair per quarter of the chunk --------------------
+    float wm = fmaxf(e, __shfl_xor_sync(0xffffffffu, e, 8));
+    wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, 16));
+    const float t = live ? __expf(e - wm) : 0.f;
+    float ws = t + __shfl_xor_sync(0xffffffffu, t, 8);
+    ws += __shfl_xor_sync(0xffffffffu, ws, 16);
+    COBS_ACC(5);
+    if (live) __stcg(p.e + ((size_t)u * G + i) * NB + blk, t);
+    if (bl == 0 && i < G) __stcg(reinterpret_cast<float2 *>(p.lse_part) + (((size_t)u * G + i) * cpu + ck) * 4 + q, make_float2(wm, ws));
+    COBS_ACC(6);
+    if (pend_u != u) flush();
+    pend_u = u;
+    ++pend_n;
+    ++n;
+    ++j;
+    COBS_ACC(7);
+  }
+  flush();
+  COBS_ACC_FLUSH(400 + (int)blockIdx.x * 8 + warp);
+}
+
+// ---------------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------------
 template <int DT, int D, int WPT, int NT>
@@ -1174,7 +1570,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
     COBS_STAMP(3);
   } else if (phases & PH_SCORE) {
     // ---- selection team ----------------------------------------------------------------------------------------
-    select_team(p, seq_lens, (int)threadIdx.x - kFWarps * 32);
+    select_team<1>(p, seq_lens, (int)threadIdx.x - kFWarps * 32, 1, 1);
   }
   // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
   __syncthreads();
@@ -1187,6 +1583,71 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
   if (is_last) {
     const int units = p.B * p.Hkv;
     for (int i = threadIdx.x; i < units; i += kFThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
+    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; }
+  }
+}
+
+// The step with phase S on tcgen05 (packed E2M1, full key space, D = 128, r = 8); phases must include PH_SCORE.
+__global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p, int phases, const __grid_constant__ CUtensorMap tmap_xi) {
+  extern __shared__ unsigned char fsm_raw[];
+  __shared__ __align__(8) uint64_t ubar[kBCount];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  __shared__ int s_len[kLenCache];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wg = blockIdx.x * kFWarps + warp, n_wg = gridDim.x * kFWarps;
+  unsigned char *fsm = fsm_raw + ((1024u - ((uint32_t)__cvta_generic_to_shared(fsm_raw) & 1023u)) & 1023u);
+  const uint32_t bars = (uint32_t)__cvta_generic_to_shared(ubar);
+  const int *seq_lens = p.seq_lens;
+  if (p.B <= kLenCache) {
+    for (int i = threadIdx.x; i < p.B; i += kUThreads) s_len[i] = p.seq_lens[i];
+    seq_lens = s_len;
+  }
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kUStages; ++i) { mbar_init(bars + (kBFull + i) * 8, 1); mbar_init(bars + (kBEmpty + i) * 8, 5); }
+    for (int i = 0; i < kUAccBufs; ++i) { mbar_init(bars + (kBTFull + i) * 8, 1); mbar_init(bars + (kBTEmpty + i) * 8, 4); }
+    for (int i = 0; i < kUTiles; ++i) mbar_init(bars + (kBQFull + i) * 8, 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == kFWarps + kSelWarps + 1) {       // the MMA warp owns the tensor memory
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(&s_tmem)), "r"(kUAccCols * kUAccBufs));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int *abort_flag = &s_abort;
+  if (warp < kFWarps) {
+    umma_epilogue(p, seq_lens, fsm, bars, tmem, warp, lane, abort_flag);
+    // every streaming warp is done with the scoring stages before any of them reuses the memory for attention
+    asm volatile("bar.sync 4, %0;\n" ::"n"(kFWarps * 32) : "memory");
+    if (phases & PH_ATTEND) attend_phase<128>(p, seq_lens, fsm + warp * kWarpSmemBytes, wg, n_wg, lane, true);
+  } else if (warp < kFWarps + kSelWarps) {
+    select_team<4>(p, seq_lens, (int)threadIdx.x - kFWarps * 32, 4, 0);
+  } else if (warp == kFWarps + kSelWarps) {
+    umma_producer(p, seq_lens, fsm, bars, &tmap_xi, lane, abort_flag);
+  } else if (lane == 0) {
+    umma_issuer(p, seq_lens, fsm, bars, tmem, abort_flag);
+  }
+  // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
+  tc_fence_before();
+  __syncthreads();
+  __shared__ int is_last;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    is_last = (atomicAdd(p.ctl_done, 1) + 1 == (int)gridDim.x);
+  }
+  if (warp == kFWarps + kSelWarps + 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kUAccCols * kUAccBufs));
+  }
+  __syncthreads();
+  if (is_last) {
+    const int units = p.B * p.Hkv;
+    for (int i = threadIdx.x; i < units; i += kUThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
     if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; }
   }
 }
@@ -1248,6 +1709,69 @@ bool fused_score_supported(const Params &p) {
   return false;
 }
 
+#ifndef COBS_UMMA
+#define COBS_UMMA 0                                          // 0: keep every configuration on the mma.sync scoring path
+#endif
+
+// Whether phase S of this configuration runs on tcgen05 (see the section on it above).
+static bool umma_score_supported(const Params &p) {
+  if (!COBS_UMMA || !fused_score_supported(p)) return false;
+  if (p.summ_dtype != COBS_SUMM_FP4_E2M1 || p.u_q != nullptr) return false;
+  if (p.D != 128 || p.Ds_pad != 128 || p.r != 8 || p.G > 8) return false;
+  if (p.NB % 16 != 0 || p.NB / 16 < kUStages) return false;  // whole chunks; a unit spans more chunks than are in flight
+  if ((size_t)p.B * p.Hkv * p.NB * 8 >= (size_t)1 << 31) return false;
+  if (reinterpret_cast<uintptr_t>(p.xi) % 32 != 0 || reinterpret_cast<uintptr_t>(p.mean) % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(p.scale) % 16 != 0) return false;
+  return true;
+}
+
+typedef CUresult (*cobs_tmap_encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                        const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                        CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static cudaError_t launch_fused_umma(Params p, int phases, cudaStream_t stream) {
+  static cobs_tmap_encode_fn encode = nullptr;
+  static std::mutex mu;
+  static int grid_cache[64] = {0};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!encode) {
+      void *fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if ((e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres)) != cudaSuccess) return e;
+      if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+      encode = reinterpret_cast<cobs_tmap_encode_fn>(fn);
+    }
+    if (grid_cache[dev] == 0) {
+      if ((e = cudaFuncSetAttribute(fused_step_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUSmemBytes)) != cudaSuccess)
+        return e;
+      int sms = 0, occ = 0;
+      if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+      if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fused_step_umma_kernel, kUThreads, kUSmemBytes)) != cudaSuccess)
+        return e;
+      if (occ < 1) return cudaErrorLaunchOutOfResources;
+      grid_cache[dev] = sms;                                  // one CTA per SM: the CTA holds the SM's tensor memory columns it asks for
+    }
+  }
+  // the factor rows as a 2-D tensor [rows][128 codes]; the element type makes the copy engine unpack 16 codes
+  // (8 bytes) into a 16-byte slot, which is what tcgen05.mma.kind::f8f6f4 reads
+  CUtensorMap tmap;
+  const cuuint64_t dims[2] = {128, (cuuint64_t)p.B * p.Hkv * p.NB * 8};
+  const cuuint64_t strides[1] = {64};
+  const cuuint32_t box[2] = {128, 128}, estr[2] = {1, 1};
+  if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, p.xi, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  void *args[] = {&p, &phases, &tmap};
+  e = cudaLaunchCooperativeKernel((const void *)fused_step_umma_kernel, dim3(grid_cache[dev]), dim3(kUThreads), args, kUSmemBytes, stream);
+  count_launch();
+  return e;
+}
+
 cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream) {
   if ((phases & PH_SCORE) && p.u_q) {
     Params q = p;
@@ -1256,6 +1780,7 @@ cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
+  if ((phases & PH_SCORE) && umma_score_supported(p)) return launch_fused_umma(p, phases, stream);
   const bool fp4 = p.summ_dtype == COBS_SUMM_FP4_E2M1 && (phases & PH_SCORE);
   if (!fp4) {
     return p.D == 128 ? launch_fused_t<COBS_SUMM_BF16, 128, 1, 1>(p, phases, stream)
