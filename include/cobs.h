@@ -231,6 +231,13 @@ int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void *q, const c
  * has no counterpart: it exists so that a benchmark can state how many launches a timed region held). */
 int64_t cobs_kernel_launches(void);
 
+/* Number of those launches whose scoring phase ran on the tcgen05 path (opt-in: environment variable
+ * COBS_SCORE_PATH=tcgen05, read at every call; packed E2M1 summaries in the full key space with head_dim 128,
+ * rank 8, max_blocks a multiple of 32; any other configuration, or a grid whose CTAs would meet more units than
+ * the kernel keeps query operands for, silently takes the default path).  Same results as the default path to
+ * rounding; lets a test state which path it exercised.  The paper has no counterpart. */
+int64_t cobs_tcgen05_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,7 @@ SCALE_DTYPES = {"fp32": 0, "fp16": 1}
 EXPORTS = [
     "cobs_status_string", "cobs_padded_sub_dim", "cobs_summary_bytes", "cobs_workspace_bytes", "cobs_reset_status",
     "cobs_read_status", "cobs_build_summaries", "cobs_quantise_xi", "cobs_score_select", "cobs_sparse_decode",
-    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_sparse_decode_static",
+    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_tcgen05_launches", "cobs_sparse_decode_static",
 ]
 
 
@@ -64,12 +64,17 @@ def lib():
         for name in EXPORTS[1:]:
             getattr(l, name).restype = C.c_int32
         l.cobs_kernel_launches.restype = C.c_int64
+        l.cobs_tcgen05_launches.restype = C.c_int64
         _lib = l
     return _lib
 
 
 def cobs_kernel_launches() -> int:
     return int(lib().cobs_kernel_launches())
+
+
+def cobs_tcgen05_launches() -> int:
+    return int(lib().cobs_tcgen05_launches())
 
 
 def status_string(status: int) -> str:

@@ -9,6 +9,8 @@
 namespace cobs {
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+static std::atomic<long long> g_tc_launches{0};
+void count_tcgen05_launch() { g_tc_launches.fetch_add(1, std::memory_order_relaxed); }
 
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_select(const Params &p, cudaStream_t stream);
@@ -196,6 +198,7 @@ const char *cobs_status_string(int32_t s) {
 }
 
 int64_t cobs_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+int64_t cobs_tcgen05_launches(void) { return g_tc_launches.load(std::memory_order_relaxed); }
 
 int32_t cobs_padded_sub_dim(const cobs_config *cfg) {
   if (validate_config(cfg) != COBS_OK) return -1;

@@ -51,6 +51,7 @@ struct Params {
 
 // host-side count of kernel launches (see cobs_kernel_launches)
 void count_launch(int n = 1);
+void count_tcgen05_launch();
 
 __device__ __forceinline__ void report(int32_t *status, int code) {
   if (status) atomicCAS(status, 0, code);

@@ -37,6 +37,8 @@
 #include <cuda.h>
 #include <cuda_fp8.h>
 
+#include <cstdlib>
+#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -1191,21 +1193,50 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
 // sets taking alternate chunks (warp w reads the TMEM lanes 32 (w mod 4) ..., i.e. blocks 4 (w mod 4) ... of the
 // chunk), warps 8-11 = the selection team as before.  All hand-offs are mbarriers with bounded waits.
 // ---------------------------------------------------------------------------------------------------
-constexpr int kUStages = 9;                                   // chunks in flight per CTA
-constexpr int kUStageBytes = 21504;                           // 16384 unpacked factor rows + 4096 means + 512 scales, padded to 1 KiB
-constexpr int kUMeanOff = 16384, kUScaleOff = 20480;
-constexpr int kUTiles = 4;                                    // query operands (one per unit) kept at a time
-constexpr int kUTileBytes = 5120;                             // 2048 operand tile + 2048 bf16 query rows + head factors
-constexpr int kUTileQOff = 2048, kUTileFOff = 4096;
-constexpr int kUTilesOff = kUStages * kUStageBytes;           // 193536
+constexpr int kUBlocks = 32;                                  // blocks per pipeline stage: two 128-row products
+constexpr int kUStages = 4;                                   // stages per CTA (two groups of kUAccBufs)
+constexpr int kUStageBytes = 43008;                           // 32768 unpacked factor rows + 8192 means + 1024 scales + header, padded to 1 KiB
+constexpr int kUMeanOff = 32768, kUScaleOff = 40960, kUHdrOff = 41984;
+constexpr int kUTiles = 10;                                   // query operands (one per unit the CTA meets)
+constexpr int kUTileBytes = 2048;
+constexpr int kUTilesOff = kUStages * kUStageBytes;           // 172032
+constexpr int kUFacOff = kUTilesOff + kUTiles * kUTileBytes;  // [tile][8] head factors
 constexpr int kUSmemBytes = kFusedSmemBytes + 1024;           // + slack to align the base to 1 KiB
-static_assert(kUTilesOff + kUTiles * kUTileBytes <= kFusedSmemBytes, "tcgen05 scoring layout exceeds the CTA's shared memory");
+static_assert(kUFacOff + kUTiles * 32 <= kFusedSmemBytes, "tcgen05 scoring layout exceeds the CTA's shared memory");
 constexpr int kUThreads = (kFWarps + kSelWarps + 2) * 32;     // + producer warp + MMA warp
-constexpr int kUAccCols = 16, kUAccBufs = 4;                  // tensor memory: 64 columns
-constexpr int kUWaitLimit = 2000000;                          // bounded mbarrier waits (try_wait iterations)
+constexpr int kUAccCols = 32, kUAccBufs = 2;                  // tensor memory: 2 buffers x (2 products x 16 columns)
+constexpr int kUWaitLimit = 200000;                           // bounded mbarrier waits (try_wait iterations)
+constexpr int kUMaxWaves = 8;
+static_assert(kWaves <= kUMaxWaves, "wave table too small");
+static_assert(kUStages == 2 * kUAccBufs, "a producer step and an issuer step cover the same kUAccBufs list positions");
 // mbarrier indices
 constexpr int kBFull = 0, kBEmpty = kBFull + kUStages, kBTFull = kBEmpty + kUStages, kBTEmpty = kBTFull + kUAccBufs,
-              kBQFull = kBTEmpty + kUAccBufs, kBCount = kBQFull + kUTiles;
+              kBTiles = kBTEmpty + kUAccBufs, kBCount = kBTiles + 1;
+
+// The CTA's stage list: wave by wave, a contiguous range of each wave's 32-block pieces.  Position n of the list
+// goes through pipeline slot n mod kUStages and accumulator n mod kUAccBufs whether or not it holds summarised
+// blocks (an empty position passes as a bubble), so every role can address the list at random.  The units the
+// ranges touch are numbered in list order: that number is the unit's query-operand tile.
+struct UmmaList {
+  int n_waves, total, cpu, n_tiles;
+  int len[kUMaxWaves], start[kUMaxWaves], tile0[kUMaxWaves];
+};
+__host__ __device__ inline void umma_list_make(UmmaList &l, int units, int NB, int grid, int bid) {
+  l.cpu = NB / kUBlocks;
+  l.n_waves = (units >= 2 * kWaves) ? kWaves : 1;
+  l.total = 0;
+  l.n_tiles = 0;
+  for (int w = 0; w < l.n_waves; ++w) {
+    const int u0 = (units * w) / l.n_waves, u1 = (units * (w + 1)) / l.n_waves;
+    const int tot = (u1 - u0) * l.cpu, per = (tot + grid - 1) / grid;
+    const int c = (bid * per < tot) ? bid * per : tot, c_end = (bid * per + per < tot) ? bid * per + per : tot;
+    l.start[w] = u0 * l.cpu + c;
+    l.len[w] = c_end - c;
+    l.total += c_end - c;
+    l.tile0[w] = l.n_tiles;
+    if (c_end > c) l.n_tiles += (l.start[w] + l.len[w] - 1) / l.cpu - l.start[w] / l.cpu + 1;
+  }
+}
 
 __device__ __forceinline__ bool mbar_wait_lim(uint32_t bar, uint32_t parity) {
   for (int it = 0; it < kUWaitLimit; ++it) {
@@ -1232,187 +1263,195 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
 // D fp32, A = E2M1, B = E4M3, both K-major, M = 128, N = 16
 constexpr uint32_t kUInstrDesc = (1u << 4) | (5u << 7) | (0u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
 
-// The CTA's chunk list: wave by wave, a contiguous range of each wave's chunks, chunks past a unit's summarised
-// blocks left out.  Every role walks the same list with the same sequence numbers.
-struct UmmaIter {
-  int wave, left, u, ck, n_sum, units, cpu, n_waves;
-  __device__ void load_unit(const Params &p, const int *seq_lens) {
-    n_sum = (u < units) ? min(seq_lens[u / p.Hkv] / p.L, p.NB) : 0;
-  }
-  __device__ void open_wave(const Params &p, const int *seq_lens, int w) {
-    wave = w;
-    const int u0 = (units * w) / n_waves, u1 = (units * (w + 1)) / n_waves;
-    const int tot = (u1 - u0) * cpu, per = (tot + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int c = min((int)blockIdx.x * per, tot), c_end = min((int)blockIdx.x * per + per, tot);
-    left = c_end - c;
-    u = u0 + c / cpu;
-    ck = c - (c / cpu) * cpu;
-    load_unit(p, seq_lens);
-  }
-  __device__ void init(const Params &p, const int *seq_lens) {
-    units = p.B * p.Hkv; cpu = (p.NB + 15) / 16;
-    n_waves = (units >= 2 * kWaves) ? kWaves : 1;
-    open_wave(p, seq_lens, 0);
-  }
-  // the next chunk (unit, chunk in unit, summarised blocks of the unit); false at the end of the list
-  __device__ bool next(const Params &p, const int *seq_lens, int &ou, int &ock, int &on_sum) {
-    for (;;) {
-      if (left <= 0) {
-        if (wave + 1 >= n_waves) return false;
-        open_wave(p, seq_lens, wave + 1);
-        continue;
-      }
-      if (ck * 16 < n_sum) {
-        ou = u; ock = ck; on_sum = n_sum;
-        --left;
-        if (++ck == cpu) { ++u; ck = 0; load_unit(p, seq_lens); }
-        return true;
-      }
-      left -= cpu - ck;                          // the rest of this unit has no summaries
-      ++u; ck = 0;
-      load_unit(p, seq_lens);
-    }
-  }
-};
-
 __device__ __forceinline__ void umma_abort(const Params &p, volatile int *abort_flag, int lane) {
   if (lane == 0) { report(p.status, COBS_ERR_TIMEOUT); *abort_flag = 1; }
 }
 
-// Producer warp: keeps kUStages chunks in flight and builds the query operand of every unit the CTA meets.
-__device__ void umma_producer(const Params &p, const int *seq_lens, unsigned char *fsm, uint32_t bars, const CUtensorMap *tmap,
-                              int lane, volatile int *abort_flag) {
-  UmmaIter it;
-  it.init(p, seq_lens);
-  const int G = p.G, NB = p.NB;
-  const int scale_sz = (p.scale_dtype == COBS_SCALE_FP16) ? 2 : 4;
-  const uint32_t scale_bytes = 16 * 8 * scale_sz;
-  const uint32_t sm = (uint32_t)__cvta_generic_to_shared(fsm);
-  const float inv_sqrt_d = 1.0f / sqrtf(128.0f);
-  int n = 0, cur_u = -1, tile_seq = -1, u = 0, ck = 0, n_sum = 0;
-  COBS_ACC_DECL;
-  while (it.next(p, seq_lens, u, ck, n_sum)) {
-    if (*abort_flag) break;
-    const int slot = n % kUStages;
-    COBS_ACC(0);
-    if (n >= kUStages && !mbar_wait_lim(bars + (kBEmpty + slot) * 8, ((n / kUStages) - 1) & 1)) { umma_abort(p, abort_flag, lane); break; }
-    COBS_ACC(1);
-    if (u != cur_u) {
-      // ---- query operand of unit u: rows h (high E4M3 term) and 8 + h (remainder), 128-byte swizzled ----------
-      cur_u = u;
-      ++tile_seq;
-      unsigned char *tile = fsm + kUTilesOff + (tile_seq & (kUTiles - 1)) * kUTileBytes;
+// Query operand of one unit, built by one warp: rows h (high E4M3 term) and 8 + h (remainder) of a 16 x 128
+// operand, 128-byte swizzled, plus the head factors (power of two that was divided out, times 1/sqrt(D)).
+__device__ void umma_build_tile(const Params &p, unsigned char *fsm, int t, int u, int lane) {
+  unsigned char *tile = fsm + kUTilesOff + t * kUTileBytes;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) reinterpret_cast<uint4 *>(tile)[lane * 4 + j] = make_uint4(0, 0, 0, 0);
-      __syncwarp();
-      const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
-      for (int g = 0; g < G; ++g) {
-        const __nv_bfloat16 *qrow = p.q + ((size_t)b_idx * p.Hq + h * G + g) * 128;
-        const uint2 raw = *reinterpret_cast<const uint2 *>(qrow + 4 * lane);
-        const float x0 = bf16_lo(raw.x), x1 = bf16_hi(raw.x), x2 = bf16_lo(raw.y), x3 = bf16_hi(raw.y);
-        const float mx = warp_max(fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3))));
-        int ex = 0;
-        if (mx > 0.f) frexpf(mx, &ex);
-        const float sc = ldexpf(1.0f, 8 - ex);               // largest |q| of the head lands in [128, 256)
-        const float y0 = x0 * sc, y1 = x1 * sc, y2 = x2 * sc, y3 = x3 * sc;
-        const __nv_fp8x2_storage_t h01 = __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);
-        const __nv_fp8x2_storage_t h23 = __nv_cvt_float2_to_fp8x2(make_float2(y2, y3), __NV_SATFINITE, __NV_E4M3);
-        const __half2_raw b01 = __nv_cvt_fp8x2_to_halfraw2(h01, __NV_E4M3), b23 = __nv_cvt_fp8x2_to_halfraw2(h23, __NV_E4M3);
-        const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&b01));
-        const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&b23));
-        const __nv_fp8x2_storage_t l01 = __nv_cvt_float2_to_fp8x2(make_float2(y0 - f01.x, y1 - f01.y), __NV_SATFINITE, __NV_E4M3);
-        const __nv_fp8x2_storage_t l23 = __nv_cvt_float2_to_fp8x2(make_float2(y2 - f23.x, y3 - f23.y), __NV_SATFINITE, __NV_E4M3);
-        const uint32_t hi4 = (uint32_t)h01 | ((uint32_t)h23 << 16), lo4 = (uint32_t)l01 | ((uint32_t)l23 << 16);
-        const int kb = 4 * lane;                            // byte (= element) position in the row
-        const int nh = g, nl = 8 + g;
-        *reinterpret_cast<uint32_t *>(tile + (nh >> 3) * 1024 + (nh & 7) * 128 + (((kb >> 4) ^ (nh & 7)) << 4) + (kb & 15)) = hi4;
-        *reinterpret_cast<uint32_t *>(tile + (nl >> 3) * 1024 + (nl & 7) * 128 + (((kb >> 4) ^ (nl & 7)) << 4) + (kb & 15)) = lo4;
-        *reinterpret_cast<uint2 *>(tile + kUTileQOff + g * 256 + lane * 8) = raw;
-        if (lane == 0) reinterpret_cast<float *>(tile + kUTileFOff)[g] = ldexpf(1.0f, ex - 8) * inv_sqrt_d;
-      }
-      fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bars + (kBQFull + (tile_seq & (kUTiles - 1))) * 8);
+  for (int j = 0; j < 4; ++j) reinterpret_cast<uint4 *>(tile)[lane * 4 + j] = make_uint4(0, 0, 0, 0);
+  __syncwarp();
+  const int G = p.G, b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
+  const float inv_sqrt_d = 1.0f / sqrtf(128.0f);
+  uint2 raws[8];                                            // all heads' loads in flight together
+#pragma unroll
+  for (int g = 0; g < 8; ++g)
+    raws[g] = (g < G) ? *reinterpret_cast<const uint2 *>(p.q + ((size_t)b_idx * p.Hq + h * G + g) * 128 + 4 * lane) : make_uint2(0, 0);
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    if (g >= G) break;
+    const uint2 raw = raws[g];
+    const float x0 = bf16_lo(raw.x), x1 = bf16_hi(raw.x), x2 = bf16_lo(raw.y), x3 = bf16_hi(raw.y);
+    const float mx = warp_max(fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3))));
+    int ex = 0;
+    if (mx > 0.f) frexpf(mx, &ex);
+    const float sc = ldexpf(1.0f, 8 - ex);                   // largest |q| of the head lands in [128, 256)
+    const float y0 = x0 * sc, y1 = x1 * sc, y2 = x2 * sc, y3 = x3 * sc;
+    const __nv_fp8x2_storage_t h01 = __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);
+    const __nv_fp8x2_storage_t h23 = __nv_cvt_float2_to_fp8x2(make_float2(y2, y3), __NV_SATFINITE, __NV_E4M3);
+    const __half2_raw b01 = __nv_cvt_fp8x2_to_halfraw2(h01, __NV_E4M3), b23 = __nv_cvt_fp8x2_to_halfraw2(h23, __NV_E4M3);
+    const float2 f01 = __half22float2(*reinterpret_cast<const __half2 *>(&b01));
+    const float2 f23 = __half22float2(*reinterpret_cast<const __half2 *>(&b23));
+    const __nv_fp8x2_storage_t l01 = __nv_cvt_float2_to_fp8x2(make_float2(y0 - f01.x, y1 - f01.y), __NV_SATFINITE, __NV_E4M3);
+    const __nv_fp8x2_storage_t l23 = __nv_cvt_float2_to_fp8x2(make_float2(y2 - f23.x, y3 - f23.y), __NV_SATFINITE, __NV_E4M3);
+    const uint32_t hi4 = (uint32_t)h01 | ((uint32_t)h23 << 16), lo4 = (uint32_t)l01 | ((uint32_t)l23 << 16);
+    const int kb = 4 * lane;                                // byte (= element) position in the row
+    const int nh = g, nl = 8 + g;
+    *reinterpret_cast<uint32_t *>(tile + (nh >> 3) * 1024 + (nh & 7) * 128 + (((kb >> 4) ^ (nh & 7)) << 4) + (kb & 15)) = hi4;
+    *reinterpret_cast<uint32_t *>(tile + (nl >> 3) * 1024 + (nl & 7) * 128 + (((kb >> 4) ^ (nl & 7)) << 4) + (kb & 15)) = lo4;
+    if (lane == 0) reinterpret_cast<float *>(fsm + kUFacOff)[t * 8 + g] = ldexpf(1.0f, ex - 8) * inv_sqrt_d;
+  }
+}
+
+// All query operands of the CTA's list, built by the selection team's warps before they have anything to select.
+__device__ void umma_build_tiles(const Params &p, const UmmaList &l, unsigned char *fsm, uint32_t bars, int team_warp, int lane) {
+  for (int w = 0; w < l.n_waves; ++w) {
+    if (l.len[w] <= 0) continue;
+    const int uf = l.start[w] / l.cpu, ul = (l.start[w] + l.len[w] - 1) / l.cpu;
+    for (int u = uf + team_warp; u <= ul; u += kSelWarps) umma_build_tile(p, fsm, l.tile0[w] + (u - uf), u, lane);
+  }
+  fence_proxy_async();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bars + kBTiles * 8);
+}
+
+// Producer warp.  Step k of the warp issues the list positions kUAccBufs k ... together: lane a does the
+// arithmetic of position kUAccBufs k + a and writes the slot's 16-byte header {unit, 32-block piece, summarised
+// blocks, flags | tile} for the other roles; lane 0 then issues the copies (their operands are warp-uniform):
+// 256 factor rows (tensor copy, unpacked by the copy engine), 32 means, 32 x 8 scales.
+__device__ void umma_producer(const Params &p, const int *seq_lens, const UmmaList &l, unsigned char *fsm, uint32_t bars,
+                              const CUtensorMap *tmap, int lane, volatile int *abort_flag) {
+  const int NB = p.NB, cpu = l.cpu;
+  const int scale_sz = (p.scale_dtype == COBS_SCALE_FP16) ? 2 : 4;
+  const uint32_t scale_bytes = kUBlocks * 8 * scale_sz;
+  const uint32_t sm = (uint32_t)__cvta_generic_to_shared(fsm);
+  int w = 0, o = lane;
+  COBS_ACC_DECL;
+  for (int k = 0;; ++k) {
+    while (w < l.n_waves && o >= l.len[w]) { o -= l.len[w]; ++w; }
+    const int slot = (lane & (kUAccBufs - 1)) + kUAccBufs * (k & 1);
+    const bool has = lane < kUAccBufs && w < l.n_waves;
+    if (!__any_sync(0xffffffffu, has) || *abort_flag) break;
+    int u = 0, ck = 0, n_sum = 0, tile = 0;
+    bool valid = false;
+    if (has) {
+      const int c = l.start[w] + o;
+      u = c / cpu; ck = c - u * cpu;
+      n_sum = min(seq_lens[u / p.Hkv] / p.L, NB);
+      valid = ck * kUBlocks < n_sum;
+      tile = l.tile0[w] + (u - l.start[w] / cpu);
     }
-    {
-      // lane 0: the factor rows (tensor copy); lanes 1 and 2: the means and the scales (one bulk-copy instruction)
-      const uint32_t st = sm + slot * kUStageBytes, bar = bars + (kBFull + slot) * 8;
-      const uint32_t rec0 = (uint32_t)(u * NB + ck * 16);        // < 2^28 (checked on the host)
-      if (lane == 0) {
-        mbar_expect_tx(bar, 8192u + 4096u + scale_bytes);
-        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-                     ::"r"(st), "l"(tmap), "r"(0), "r"((int)(rec0 * 8u)), "r"(bar) : "memory");
-      } else if (lane < 3) {
-        const bool is_mean = lane == 1;
-        const char *src = is_mean ? (const char *)p.mean + (size_t)rec0 * 256 : (const char *)p.scale + (size_t)rec0 * (8 * scale_sz);
-        bulk_g2s(st + (is_mean ? kUMeanOff : kUScaleOff), src, is_mean ? 4096u : scale_bytes, bar);
-      }
-    }
+    COBS_ACC(0);
+    bool ok = true;
+    if (has && k > 1) ok = mbar_wait_lim(bars + (kBEmpty + slot) * 8, ((k >> 1) - 1) & 1);
+    if (!__all_sync(0xffffffffu, ok)) { umma_abort(p, abort_flag, lane); break; }
+    COBS_ACC(1);
+    if (has) *reinterpret_cast<int4 *>(fsm + slot * kUStageBytes + kUHdrOff) = make_int4(u, ck, n_sum, (valid ? 1 : 0) | (tile << 8));
+    __syncwarp();
+    const unsigned hm = __ballot_sync(0xffffffffu, has), vm = __ballot_sync(0xffffffffu, valid);
+    const uint32_t rec0 = (uint32_t)(u * NB + ck * kUBlocks);    // < 2^28 (checked on the host)
     COBS_ACC(2);
-    ++n;
+#pragma unroll
+    for (int sl = 0; sl < kUAccBufs; ++sl) {
+      const uint32_t rec = __shfl_sync(0xffffffffu, rec0, sl);
+      if (lane == 0 && ((hm >> sl) & 1u)) {
+        const int slot_s = sl + kUAccBufs * (k & 1);
+        const uint32_t st = sm + slot_s * kUStageBytes, bar = bars + (kBFull + slot_s) * 8;
+        if ((vm >> sl) & 1u) {
+          mbar_expect_tx(bar, (uint32_t)(kUBlocks * 8 * 64) + (uint32_t)(kUBlocks * 256) + scale_bytes);
+          asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+                       ::"r"(st), "l"(tmap), "r"(0), "r"((int)(rec * 8u)), "r"(bar) : "memory");
+          bulk_g2s(st + kUMeanOff, (const char *)p.mean + (size_t)rec * 256, (uint32_t)(kUBlocks * 256), bar);
+          bulk_g2s(st + kUScaleOff, (const char *)p.scale + (size_t)rec * (8 * scale_sz), scale_bytes, bar);
+        } else {
+          mbar_arrive(bar);                       // a bubble: nothing to copy
+        }
+      }
+    }
+    COBS_ACC(3);
+    o += kUAccBufs;
   }
   COBS_ACC_FLUSH((int)blockIdx.x);
 }
 
-// MMA issuer (one thread): one 128 x 16 x 128 product per chunk into the next accumulator buffer.
-__device__ void umma_issuer(const Params &p, const int *seq_lens, unsigned char *fsm, uint32_t bars, uint32_t tmem,
+// MMA issuer warp.  Lane a < kUAccBufs waits for and decodes the list positions a, a + kUAccBufs, ... (accumulator
+// buffer a); lane 0 issues: two 128 x 16 x 128 products (four K steps each) per stage, then one commit that hands
+// the accumulators to the epilogue.  A bubble passes its barrier on by hand.
+__device__ void umma_issuer(const Params &p, const UmmaList &l, unsigned char *fsm, uint32_t bars, uint32_t tmem, int lane,
                             volatile int *abort_flag) {
-  UmmaIter it;
-  it.init(p, seq_lens);
   const uint64_t desc0 = umma_desc((uint32_t)__cvta_generic_to_shared(fsm));   // the whole region lies below 2^18
-  int n = 0, cur_u = -1, tile_seq = -1, u = 0, ck = 0, n_sum = 0;
+  int n = lane;
   COBS_ACC_DECL;
-  while (it.next(p, seq_lens, u, ck, n_sum)) {
-    if (*abort_flag) break;
-    const int slot = n % kUStages, acc = n % kUAccBufs;
+  if (!mbar_wait_lim(bars + kBTiles * 8, 0)) { umma_abort(p, abort_flag, lane); return; }
+  for (int k = 0;; ++k) {
+    const int slot = (lane & (kUAccBufs - 1)) + kUAccBufs * (k & 1), fpar = (k >> 1) & 1;
+    const bool has = lane < kUAccBufs && n < l.total;
+    if (!__any_sync(0xffffffffu, has) || *abort_flag) break;
     bool ok = true;
+    int4 hdr = make_int4(0, 0, 0, 0);
     COBS_ACC(0);
-    if (u != cur_u) {
-      cur_u = u;
-      ++tile_seq;
-      ok = mbar_wait_lim(bars + (kBQFull + (tile_seq & (kUTiles - 1))) * 8, (tile_seq / kUTiles) & 1);
+    if (has) {
+      ok = mbar_wait_lim(bars + (kBFull + slot) * 8, fpar);
+      hdr = *reinterpret_cast<const int4 *>(fsm + slot * kUStageBytes + kUHdrOff);
     }
     COBS_ACC(1);
-    ok = ok && mbar_wait_lim(bars + (kBFull + slot) * 8, (n / kUStages) & 1);
+    const bool valid = has && (hdr.w & 1);
+    const int tile = (hdr.w >> 8) & 0xff;
+    if (has && ok && k > 0) ok = mbar_wait_lim(bars + (kBTEmpty + lane) * 8, (k - 1) & 1);
     COBS_ACC(2);
-    if (ok && n >= kUAccBufs) ok = mbar_wait_lim(bars + (kBTEmpty + acc) * 8, ((n / kUAccBufs) - 1) & 1);
-    COBS_ACC(3);
-    if (!ok) { umma_abort(p, abort_flag, 0); break; }
+    if (!__all_sync(0xffffffffu, ok)) { umma_abort(p, abort_flag, lane); break; }
     tc_fence_after();
-    const uint64_t da0 = desc0 + (uint64_t)((slot * kUStageBytes) >> 4);
-    const uint64_t db0 = desc0 + (uint64_t)((kUTilesOff + (tile_seq & (kUTiles - 1)) * kUTileBytes) >> 4);
+    const unsigned hm = __ballot_sync(0xffffffffu, has), vm = __ballot_sync(0xffffffffu, valid);
 #pragma unroll
-    for (int ks = 0; ks < 4; ++ks) {
-      const uint64_t da = da0 + 2 * ks, db = db0 + 2 * ks;     // 32 bytes along K per step
-      const uint32_t accum = ks > 0;
-      asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}\n"
-                   ::"r"(tmem + acc * kUAccCols), "l"(da), "l"(db), "r"(kUInstrDesc), "r"(accum) : "memory");
+    for (int a = 0; a < kUAccBufs; ++a) {
+      const int tile_a = __shfl_sync(0xffffffffu, tile, a);
+      if (lane == 0 && ((hm >> a) & 1u)) {
+        const int slot_a = a + kUAccBufs * (k & 1);
+        const uint32_t bar_t = bars + (kBTFull + a) * 8;
+        if ((vm >> a) & 1u) {
+          const uint64_t db0 = desc0 + (uint64_t)((kUTilesOff + tile_a * kUTileBytes) >> 4);
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const uint64_t da0 = desc0 + (uint64_t)((slot_a * kUStageBytes + half * 16384) >> 4);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint64_t da = da0 + 2 * ks, db = db0 + 2 * ks;   // 32 bytes along K per step
+              const uint32_t accum = ks > 0;
+              asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}\n"
+                           ::"r"(tmem + a * kUAccCols + half * 16), "l"(da), "l"(db), "r"(kUInstrDesc), "r"(accum) : "memory");
+            }
+          }
+          tc_commit(bar_t);
+        } else {
+          mbar_arrive(bar_t);
+        }
+      }
     }
-    tc_commit(bars + (kBEmpty + slot) * 8);
-    tc_commit(bars + (kBTFull + acc) * 8);
-    COBS_ACC(4);
-    ++n;
+    COBS_ACC(3);
+    n += kUAccBufs;
   }
   COBS_ACC_FLUSH(200 + (int)blockIdx.x);
 }
 
-// Epilogue warp (streaming warps 0-7; set = warp / 4 takes the chunks of its parity, warp mod 4 = TMEM lane quarter):
-// lane (bl, i) = (lane / 8, lane % 8) holds accumulator row (block 4 q + bl of the chunk, factor i).
-// Leaves per block t = exp(e - chunk max) and per chunk the (max, sum) pairs, like the mma.sync path; each warp
-// counts the chunk on the unit once, so a unit is complete at 4 x its chunks.
-__device__ void umma_epilogue(const Params &p, const int *seq_lens, unsigned char *fsm, uint32_t bars, uint32_t tmem, int warp,
+// Epilogue warp (streaming warps 0-7; set = warp / 4 takes the list positions of its parity, warp mod 4 = TMEM lane
+// quarter): lane (bl, i) = (lane / 8, lane % 8) holds, for each half of the stage, accumulator row (block
+// 16 half + 4 q + bl, factor i).  Leaves per block t = exp(e - max over the warp's four blocks of a half) and that
+// (max, sum) pair, i.e. four pairs per 16-block chunk and head; each warp counts a 16-block chunk on the unit
+// once, so a unit is complete at 4 x its chunks.
+__device__ void umma_epilogue(const Params &p, const UmmaList &l, unsigned char *fsm, uint32_t bars, uint32_t tmem, int warp,
                               int lane, volatile int *abort_flag) {
   const int set = warp >> 2, q = warp & 3;
   const int gid = lane >> 2, tig = lane & 3;      // mma.sync fragment coordinates (mean term)
   const int bl = lane >> 3, i = lane & 7;
-  const int G = p.G, NB = p.NB, cpu = (NB + 15) / 16;
+  const int G = p.G, NB = p.NB, cpu16 = NB / 16;
   const bool scale_f16 = p.scale_dtype == COBS_SCALE_FP16;
   const float inv_sqrt_d = 1.0f / sqrtf(128.0f), ln_l = logf((float)p.L);
-  UmmaIter it;
-  it.init(p, seq_lens);
-  int n = 0, j = 0, cur_u = -1, tile_seq = -1, my_u = -1, pend_u = -1, pend_n = 0, u = 0, ck = 0, n_sum = 0;
+  int my_u = -1, pend_u = -1, pend_n = 0;
   uint32_t bm[8][2];
-  float fac = 0.f;
+  float fac2 = 0.f;
 #pragma unroll
   for (int m = 0; m < 8; ++m) bm[m][0] = bm[m][1] = 0u;
   auto flush = [&]() {
@@ -1424,107 +1463,125 @@ __device__ void umma_epilogue(const Params &p, const int *seq_lens, unsigned cha
     }
   };
   COBS_ACC_DECL;
-  while (it.next(p, seq_lens, u, ck, n_sum)) {
-    if (u != cur_u) { cur_u = u; ++tile_seq; }
-    if ((n & 1) != set) { ++n; continue; }
+  if (!mbar_wait_lim(bars + kBTiles * 8, 0)) { umma_abort(p, abort_flag, lane); return; }
+  for (int n = set, j = 0; n < l.total; n += 2, ++j) {
     if (*abort_flag) break;
+    const int slot = n & (kUStages - 1), fpar = (n / kUStages) & 1, tfpar = j & 1;
+    const uint32_t bar_empty = bars + (kBEmpty + slot) * 8, bar_tfull = bars + (kBTFull + set) * 8, bar_tempty = bars + (kBTEmpty + set) * 8;
     COBS_ACC(0);
-    const int slot = n % kUStages, acc = n % kUAccBufs;
-    const unsigned char *tile = fsm + kUTilesOff + (tile_seq & (kUTiles - 1)) * kUTileBytes;
+    if (!mbar_wait_lim(bars + (kBFull + slot) * 8, fpar)) { umma_abort(p, abort_flag, lane); break; }
+    COBS_ACC(1);
+    const unsigned char *stg = fsm + slot * kUStageBytes;
+    const int4 hdr = *reinterpret_cast<const int4 *>(stg + kUHdrOff);
+    const int u = hdr.x, ck = hdr.y, n_sum = hdr.z;
+    if (!(hdr.w & 1)) {                          // a bubble: pass the barriers on
+      if (!mbar_wait_lim(bar_tfull, tfpar)) { umma_abort(p, abort_flag, lane); break; }
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(bar_empty); mbar_arrive(bar_tempty); }
+      continue;
+    }
     if (u != my_u) {
-      if (!mbar_wait_lim(bars + (kBQFull + (tile_seq & (kUTiles - 1))) * 8, (tile_seq / kUTiles) & 1)) { umma_abort(p, abort_flag, lane); break; }
+      // ---- a new unit: query fragments for the mean product (column = head gid; k order as the rows are read) ----
       my_u = u;
-      const uint32_t qs = (uint32_t)__cvta_generic_to_shared(tile + kUTileQOff);
+      const int tile = (hdr.w >> 8) & 0xff;
+      const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
+      const __nv_bfloat16 *qg = p.q + ((size_t)b_idx * p.Hq + h * G) * 128;
 #pragma unroll
       for (int m = 0; m < 4; ++m) {
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (gid < G) v = lds128(qs + gid * 256 + (tig + 4 * m) * 16);
+        if (gid < G) v = *reinterpret_cast<const uint4 *>(qg + gid * 128 + (tig + 4 * m) * 8);
         bm[2 * m][0] = v.x; bm[2 * m][1] = v.y; bm[2 * m + 1][0] = v.z; bm[2 * m + 1][1] = v.w;
       }
-      fac = (i < G) ? reinterpret_cast<const float *>(tile + kUTileFOff)[i] : 0.f;
+      const float fac = (i < G) ? reinterpret_cast<const float *>(fsm + kUFacOff)[tile * 8 + i] : 0.f;
+      fac2 = fac * fac;
     }
-    COBS_ACC(1);
-    if (!mbar_wait_lim(bars + (kBFull + slot) * 8, (n / kUStages) & 1)) { umma_abort(p, abort_flag, lane); break; }
     COBS_ACC(2);
-    const unsigned char *stg = fsm + slot * kUStageBytes;
-    // ---- first-order term of blocks 4 q .. 4 q + 3 (rows 0-3 of an m16n8k16 tile; columns = heads) ------------
+    // ---- first-order term: rows 0-3 of an m16n8k16 tile = blocks 4 q .. of half 0, rows 8-11 = those of half 1 -----
     float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;
     {
       const uint32_t ma = (uint32_t)__cvta_generic_to_shared(stg + kUMeanOff) + (4 * q + (gid & 3)) * 256 + tig * 16;
 #pragma unroll
       for (int m = 0; m < 4; ++m) {
-        uint4 va = lds128(ma + m * 64);
-        if (gid >= 4) va = make_uint4(0, 0, 0, 0);
-        mma16816_bf16(c0, c1, c2, c3, va.x, 0u, va.y, 0u, bm[2 * m][0], bm[2 * m][1]);
-        mma16816_bf16(e0, e1, e2, e3, va.z, 0u, va.w, 0u, bm[2 * m + 1][0], bm[2 * m + 1][1]);
+        uint4 va = lds128(ma + m * 64), vb = lds128(ma + 16 * 256 + m * 64);
+        if (gid >= 4) { va = make_uint4(0, 0, 0, 0); vb = va; }
+        mma16816_bf16(c0, c1, c2, c3, va.x, vb.x, va.y, vb.y, bm[2 * m][0], bm[2 * m][1]);
+        mma16816_bf16(e0, e1, e2, e3, va.z, vb.z, va.w, vb.w, bm[2 * m + 1][0], bm[2 * m + 1][1]);
       }
     }
-    const float f0 = (c0 + e0) * inv_sqrt_d, f1 = (c1 + e1) * inv_sqrt_d;     // lane (gid < 4, tig): block 4q+gid, heads 2tig, 2tig+1
-    const int srow = (4 * q + bl) * 8 + i;
-    const float sc = scale_f16 ? __half2float(reinterpret_cast<const __half *>(stg + kUScaleOff)[srow])
-                               : reinterpret_cast<const float *>(stg + kUScaleOff)[srow];
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bars + (kBEmpty + slot) * 8);      // this warp is done with the stage
-    // ---- the chunk's product from tensor memory ---------------------------------------------------------------
+    // lane (gid < 4, tig): block 4 q + gid of each half, heads 2 tig and 2 tig + 1
+    const float fm[2][2] = {{(c0 + e0) * inv_sqrt_d, (c1 + e1) * inv_sqrt_d}, {(c2 + e2) * inv_sqrt_d, (c3 + e3) * inv_sqrt_d}};
+    float sc[2];
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const int srow = (16 * hf + 4 * q + bl) * 8 + i;
+      sc[hf] = scale_f16 ? __half2float(reinterpret_cast<const __half *>(stg + kUScaleOff)[srow])
+                         : reinterpret_cast<const float *>(stg + kUScaleOff)[srow];
+    }
     COBS_ACC(3);
-    if (!mbar_wait_lim(bars + (kBTFull + acc) * 8, (n / kUAccBufs) & 1)) { umma_abort(p, abort_flag, lane); break; }
+    // ---- the stage's products from tensor memory ----------------------------------------------------------------
+    if (!mbar_wait_lim(bar_tfull, tfpar)) { umma_abort(p, abort_flag, lane); break; }
     COBS_ACC(4);
     tc_fence_after();
-    uint32_t r[16];
+    uint32_t r[32];
     {
-      const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + acc * kUAccCols;
-      asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + set * kUAccCols;
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                   "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
                    : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                     "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                     "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                     "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                     "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                    : "r"(taddr));
       asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
     }
     tc_fence_before();
     __syncwarp();
-    if (lane == 0) mbar_arrive(bars + (kBTEmpty + acc) * 8);
-    float v[8];
+    if (lane == 0) { mbar_arrive(bar_empty); mbar_arrive(bar_tempty); }   // stage and accumulator may be refilled
+    float ssum[2];
 #pragma unroll
-    for (int h = 0; h < 8; ++h) {
-      const float x = (__uint_as_float(r[h]) + __uint_as_float(r[8 + h])) * sc;
-      v[h] = x * x;
-    }
-    // sum over the 8 factors of a block, transposing as it goes: lane i ends with head i
+    for (int hf = 0; hf < 2; ++hf) {
+      float v[8];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float keep = (i & 4) ? v[k + 4] : v[k], send = (i & 4) ? v[k] : v[k + 4];
-      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-    }
+      for (int h = 0; h < 8; ++h) {
+        const float x = (__uint_as_float(r[16 * hf + h]) + __uint_as_float(r[16 * hf + 8 + h])) * sc[hf];
+        v[h] = x * x;
+      }
+      // sum over the 8 factors of a block, transposing as it goes: lane i ends with head i
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const float keep = (i & 2) ? v[k + 2] : v[k], send = (i & 2) ? v[k] : v[k + 2];
-      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-    }
-    float ssum;
-    {
+      for (int k = 0; k < 4; ++k) {
+        const float keep = (i & 4) ? v[k + 4] : v[k], send = (i & 4) ? v[k] : v[k + 4];
+        v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+      }
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const float keep = (i & 2) ? v[k + 2] : v[k], send = (i & 2) ? v[k] : v[k + 2];
+        v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+      }
       const float keep = (i & 1) ? v[1] : v[0], send = (i & 1) ? v[0] : v[1];
-      ssum = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+      ssum[hf] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
     }
     const int src = bl * 4 + (i >> 1);
-    const float fa = __shfl_sync(0xffffffffu, f0, src), fb = __shfl_sync(0xffffffffu, f1, src);
-    const int blk = ck * 16 + 4 * q + bl;
-    const bool live = (i < G) && (blk < n_sum);
-    const float e = live ? ln_l + ((i & 1) ? fb : fa) + 0.5f * (fac * fac) * ssum : -INFINITY;
-    // ---- max and sum per head over the warp's four blocks: one pair per quarter of the chunk --------------------
-    float wm = fmaxf(e, __shfl_xor_sync(0xffffffffu, e, 8));
-    wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, 16));
-    const float t = live ? __expf(e - wm) : 0.f;
-    float ws = t + __shfl_xor_sync(0xffffffffu, t, 8);
-    ws += __shfl_xor_sync(0xffffffffu, ws, 16);
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const float fa = __shfl_sync(0xffffffffu, fm[hf][0], src), fb = __shfl_sync(0xffffffffu, fm[hf][1], src);
+      const int blk = ck * kUBlocks + 16 * hf + 4 * q + bl;
+      const bool live = (i < G) && (blk < n_sum);
+      const float e = live ? ln_l + ((i & 1) ? fb : fa) + 0.5f * fac2 * ssum[hf] : -INFINITY;
+      // max and sum per head over the warp's four blocks: one pair per quarter of a 16-block chunk
+      float wm = fmaxf(e, __shfl_xor_sync(0xffffffffu, e, 8));
+      wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, 16));
+      const float t = live ? __expf(e - wm) : 0.f;
+      float ws = t + __shfl_xor_sync(0xffffffffu, t, 8);
+      ws += __shfl_xor_sync(0xffffffffu, ws, 16);
+      if (live) __stcg(p.e + ((size_t)u * G + i) * NB + blk, t);
+      if (bl == 0 && i < G && (2 * ck + hf) * 16 < n_sum)
+        __stcg(reinterpret_cast<float2 *>(p.lse_part) + (((size_t)u * G + i) * cpu16 + 2 * ck + hf) * 4 + q, make_float2(wm, ws));
+    }
     COBS_ACC(5);
-    if (live) __stcg(p.e + ((size_t)u * G + i) * NB + blk, t);
-    if (bl == 0 && i < G) __stcg(reinterpret_cast<float2 *>(p.lse_part) + (((size_t)u * G + i) * cpu + ck) * 4 + q, make_float2(wm, ws));
-    COBS_ACC(6);
     if (pend_u != u) flush();
     pend_u = u;
-    ++pend_n;
-    ++n;
-    ++j;
-    COBS_ACC(7);
+    pend_n += 1 + (((2 * ck + 1) * 16 < n_sum) ? 1 : 0);
+    COBS_ACC(6);
   }
   flush();
   COBS_ACC_FLUSH(400 + (int)blockIdx.x * 8 + warp);
@@ -1594,6 +1651,7 @@ __global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p,
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ int s_len[kLenCache];
+  __shared__ UmmaList s_list;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wg = blockIdx.x * kFWarps + warp, n_wg = gridDim.x * kFWarps;
   unsigned char *fsm = fsm_raw + ((1024u - ((uint32_t)__cvta_generic_to_shared(fsm_raw) & 1023u)) & 1023u);
@@ -1604,10 +1662,11 @@ __global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p,
     seq_lens = s_len;
   }
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kUStages; ++i) { mbar_init(bars + (kBFull + i) * 8, 1); mbar_init(bars + (kBEmpty + i) * 8, 5); }
+    for (int i = 0; i < kUStages; ++i) { mbar_init(bars + (kBFull + i) * 8, 1); mbar_init(bars + (kBEmpty + i) * 8, 4); }
     for (int i = 0; i < kUAccBufs; ++i) { mbar_init(bars + (kBTFull + i) * 8, 1); mbar_init(bars + (kBTEmpty + i) * 8, 4); }
-    for (int i = 0; i < kUTiles; ++i) mbar_init(bars + (kBQFull + i) * 8, 1);
+    mbar_init(bars + kBTiles * 8, kSelWarps);
     s_abort = 0;
+    umma_list_make(s_list, p.B * p.Hkv, p.NB, (int)gridDim.x, (int)blockIdx.x);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == kFWarps + kSelWarps + 1) {       // the MMA warp owns the tensor memory
@@ -1621,16 +1680,21 @@ __global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p,
   const uint32_t tmem = s_tmem;
   volatile int *abort_flag = &s_abort;
   if (warp < kFWarps) {
-    umma_epilogue(p, seq_lens, fsm, bars, tmem, warp, lane, abort_flag);
+    COBS_STAMP(0);
+    umma_epilogue(p, s_list, fsm, bars, tmem, warp, lane, abort_flag);
+    COBS_STAMP(1);
     // every streaming warp is done with the scoring stages before any of them reuses the memory for attention
     asm volatile("bar.sync 4, %0;\n" ::"n"(kFWarps * 32) : "memory");
+    COBS_STAMP(2);
     if (phases & PH_ATTEND) attend_phase<128>(p, seq_lens, fsm + warp * kWarpSmemBytes, wg, n_wg, lane, true);
+    COBS_STAMP(3);
   } else if (warp < kFWarps + kSelWarps) {
+    umma_build_tiles(p, s_list, fsm, bars, warp - kFWarps, lane);
     select_team<4>(p, seq_lens, (int)threadIdx.x - kFWarps * 32, 4, 0);
   } else if (warp == kFWarps + kSelWarps) {
-    umma_producer(p, seq_lens, fsm, bars, &tmap_xi, lane, abort_flag);
-  } else if (lane == 0) {
-    umma_issuer(p, seq_lens, fsm, bars, tmem, abort_flag);
+    umma_producer(p, seq_lens, s_list, fsm, bars, &tmap_xi, lane, abort_flag);
+  } else {
+    umma_issuer(p, s_list, fsm, bars, tmem, lane, abort_flag);
   }
   // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
   tc_fence_before();
@@ -1709,16 +1773,20 @@ bool fused_score_supported(const Params &p) {
   return false;
 }
 
-#ifndef COBS_UMMA
-#define COBS_UMMA 0                                          // 0: keep every configuration on the mma.sync scoring path
-#endif
+// The tcgen05 scoring path is parity-tested but, as measured, not faster than the mma.sync path (its unpacked
+// 4-bit rows take twice the shared memory per byte in flight, which halves the copy depth of a bandwidth-bound
+// stream), so it is opt-in: environment variable COBS_SCORE_PATH=tcgen05, read at every call.
+static bool umma_requested() {
+  const char *v = getenv("COBS_SCORE_PATH");
+  return v != nullptr && strcmp(v, "tcgen05") == 0;
+}
 
 // Whether phase S of this configuration runs on tcgen05 (see the section on it above).
 static bool umma_score_supported(const Params &p) {
-  if (!COBS_UMMA || !fused_score_supported(p)) return false;
+  if (!umma_requested() || !fused_score_supported(p)) return false;
   if (p.summ_dtype != COBS_SUMM_FP4_E2M1 || p.u_q != nullptr) return false;
   if (p.D != 128 || p.Ds_pad != 128 || p.r != 8 || p.G > 8) return false;
-  if (p.NB % 16 != 0 || p.NB / 16 < kUStages) return false;  // whole chunks; a unit spans more chunks than are in flight
+  if (p.NB % kUBlocks != 0) return false;                    // whole 32-block stages
   if ((size_t)p.B * p.Hkv * p.NB * 8 >= (size_t)1 << 31) return false;
   if (reinterpret_cast<uintptr_t>(p.xi) % 32 != 0 || reinterpret_cast<uintptr_t>(p.mean) % 16 != 0 ||
       reinterpret_cast<uintptr_t>(p.scale) % 16 != 0) return false;
@@ -1757,18 +1825,24 @@ static cudaError_t launch_fused_umma(Params p, int phases, cudaStream_t stream) 
       grid_cache[dev] = sms;                                  // one CTA per SM: the CTA holds the SM's tensor memory columns it asks for
     }
   }
+  for (int bid = 0; bid < grid_cache[dev]; ++bid) {          // every unit a CTA meets needs its own operand tile
+    UmmaList l;
+    umma_list_make(l, p.B * p.Hkv, p.NB, grid_cache[dev], bid);
+    if (l.n_tiles > kUTiles) return cudaErrorNotSupported;
+  }
   // the factor rows as a 2-D tensor [rows][128 codes]; the element type makes the copy engine unpack 16 codes
   // (8 bytes) into a 16-byte slot, which is what tcgen05.mma.kind::f8f6f4 reads
   CUtensorMap tmap;
   const cuuint64_t dims[2] = {128, (cuuint64_t)p.B * p.Hkv * p.NB * 8};
   const cuuint64_t strides[1] = {64};
-  const cuuint32_t box[2] = {128, 128}, estr[2] = {1, 1};
+  const cuuint32_t box[2] = {128, kUBlocks * 8}, estr[2] = {1, 1};
   if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, p.xi, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
   void *args[] = {&p, &phases, &tmap};
   e = cudaLaunchCooperativeKernel((const void *)fused_step_umma_kernel, dim3(grid_cache[dev]), dim3(kUThreads), args, kUSmemBytes, stream);
   count_launch();
+  count_tcgen05_launch();
   return e;
 }
 
@@ -1780,7 +1854,10 @@ cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  if ((phases & PH_SCORE) && umma_score_supported(p)) return launch_fused_umma(p, phases, stream);
+  if ((phases & PH_SCORE) && umma_score_supported(p)) {
+    const cudaError_t e = launch_fused_umma(p, phases, stream);
+    if (e != cudaErrorNotSupported) return e;                // not supported: too many units per CTA, or no encoder
+  }
   const bool fp4 = p.summ_dtype == COBS_SUMM_FP4_E2M1 && (phases & PH_SCORE);
   if (!fp4) {
     return p.D == 128 ? launch_fused_t<COBS_SUMM_BF16, 128, 1, 1>(p, phases, stream)

@@ -148,6 +148,31 @@ def test_cfg4_full_size_sampled_units():
     run_stage_s(wl, inp_dev=inp, units=[(0, 0), (7, 3), (15, 7)], summ=summ)
 
 
+# --- the opt-in tcgen05 scoring path ------------------------------------------------------------------------
+
+@pytest.mark.parametrize("case", ["cfg2_32k_fp4_rank8", "cfg4_reduced", "ragged_g8_fp16_scales"])
+def test_tcgen05_scoring_path(case, monkeypatch):
+    """Same parity bar with phase S on tcgen05 (TMA-unpacked E2M1 rows x two-term E4M3 query, TMEM accumulators)."""
+    B = _binding()
+    if case == "cfg2_32k_fp4_rank8":
+        wl = WL["cfg2_32k"].replace(summary_dtype="fp4", rank=8)
+    elif case == "cfg4_reduced":
+        wl = WL["cfg4_128k"].replace(batch=3, seq_len=16384)
+    else:
+        lens = [64 * 40 + 5, 64 * 96, 100, 64 * 33]
+        wl = synth.Workload("ragged_tc", len(lens), 16, 2, 128, 64 * 96, 64, 16, rank=8, topk=12, window=200,
+                            summary_dtype="fp4", scale_dtype="fp16", key_model="block_offset", planted=2,
+                            shuffle_pages=True, seed=21, seq_lens=lens)
+    monkeypatch.setenv("COBS_SCORE_PATH", "tcgen05")
+    before = B.cobs_tcgen05_launches()
+    run_stage_s(wl)
+    assert B.cobs_tcgen05_launches() >= before + 2      # cobs_score_select and cobs_decode_step both took it
+    monkeypatch.delenv("COBS_SCORE_PATH")
+    before = B.cobs_tcgen05_launches()
+    run_stage_s(wl, units=[(0, 0)])
+    assert B.cobs_tcgen05_launches() == before          # and the default path does not
+
+
 # --- shapes and edge cases ---------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("summary_dtype,scale_dtype", [("fp32", "fp32"), ("bf16", "fp32"), ("fp4", "fp32"),
