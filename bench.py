@@ -238,6 +238,33 @@ def run_ours(args):
         torch.cuda.synchronize()
     e2e_s = max(e2e_s - (time.perf_counter() - t0), 1e-9)
 
+    # ---- optional: consecutive decode steps (append a token, rebuild a block's summary when it fills, step) ----
+    loop_info = None
+    if args.decode_loop > 0:
+        from paper_2607_09052_b200.decode_loop import DecodeLoop
+        n_loop = args.decode_loop
+        start_len = wl.seq_len - n_loop - 7                  # not a multiple of the block size; ends below capacity
+        inp["seq_lens"].fill_(start_len)
+        loop = DecodeLoop(wl.replace(seq_lens=[start_len] * nb), inp, summ=summ, ws=ws)
+        gen = torch.Generator(device=dev).manual_seed(1234)
+        pool = [(torch.randn((nb, hq, D), generator=gen, device=dev).to(torch.bfloat16),
+                 torch.randn((nb, hkv, D), generator=gen, device=dev).to(torch.bfloat16),
+                 torch.randn((nb, hkv, D), generator=gen, device=dev).to(torch.bfloat16)) for _ in range(8)]
+        ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev_a.record(stream)
+        for i in range(n_loop):
+            q_i, k_i, v_i = pool[i % len(pool)]
+            loop.step(q_i, k_i, v_i, out, None, sel, cnt)
+        ev_b.record(stream)
+        torch.cuda.synchronize()
+        if B.cobs_read_status(ws) != 0:
+            raise RuntimeError("device status after the decode loop")
+        loop_info = {"steps": n_loop, "start_len": start_len, "rebuilds": loop.rebuilds,
+                     "us_per_step_amortised": round(ev_a.elapsed_time(ev_b) * 1e3 / n_loop, 2),
+                     "note": "append + summary rebuild of the block that filled (one launch per block boundary, all "
+                             "sequences) + fused step, back to back on one stream, no L2 flush between steps"}
+
     total_ms, e2e_s = shard.job_times([total_ms, e2e_s], device=dev)   # the job is as slow as its slowest rank
     ms_per_step = total_ms / args.steps
     if rank != 0:
@@ -282,6 +309,8 @@ def run_ours(args):
         "build_summaries_ms": round(build_ms, 3),
         "wall_s_timed_region": round(wall_s, 4),
     }
+    if loop_info:
+        line["decode_loop"] = loop_info
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl, record, budget_s=20.0)
     print(json.dumps(line), flush=True)
@@ -390,6 +419,9 @@ def main():
     ap.add_argument("--seq-len", type=int, default=0, help="override the workload's context (profiling on a small case)")
     ap.add_argument("--contiguous-pages", action="store_true",
                     help="diagnostic: identity page table instead of the workload's shuffled pages")
+    ap.add_argument("--decode-loop", type=int, default=0,
+                    help="also time this many consecutive decode steps (append, rebuild on block fill, step) and "
+                         "report the amortised time per step")
     ap.add_argument("--clock-warm-s", type=float, default=0.6,
                     help="keep warming up at least this long so that the clock sampler has samples")
     args = ap.parse_args()

@@ -144,6 +144,19 @@ int32_t cobs_build_summaries(const cobs_config *cfg, const cobs_kv *kv, int32_t 
                              const cobs_summaries *out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The step before the decode step: write the new token's key and value rows (k_new, v_new: [batch][n_kv_heads][D]
+ * bf16, 16-byte aligned) at position seq_lens[b] of every sequence's paged cache and add one to seq_lens[b]
+ * (Method, Cost: a block's summary is built when the block fills, so the caller then rebuilds block
+ * seq_len / L - 1 with cobs_build_summaries whenever the new length is a multiple of L).  A sequence whose page
+ * table has no room for the position, or names a page outside [0, n_pages), leaves COBS_ERR_BOUNDS in the status
+ * word and is not touched.  Uses the first batch * 4 bytes of the workspace's staging area for a snapshot of the
+ * lengths.
+ */
+int32_t cobs_append_token(const cobs_config *cfg, const void *k_new, const void *v_new, void *k_pages, void *v_pages,
+                          const int32_t *page_table, int32_t *seq_lens, int64_t n_pages, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
+/*
  * The FP4 quantiser of step (a) on its own (Method, Quantization: E2M1, one scale per eigenvector).
  * xi_fp32 [n_vectors][Ds] -> codes [n_vectors][Ds_pad / 2] bytes, scale [n_vectors] (cfg->scale_dtype).
  *   a = max |xi_j|; scale = a / 6 (fp32 division; rounded to fp16 when the scale is fp16);

@@ -23,7 +23,7 @@ SCALE_DTYPES = {"fp32": 0, "fp16": 1}
 EXPORTS = [
     "cobs_status_string", "cobs_padded_sub_dim", "cobs_summary_bytes", "cobs_workspace_bytes", "cobs_reset_status",
     "cobs_read_status", "cobs_build_summaries", "cobs_quantise_xi", "cobs_score_select", "cobs_sparse_decode",
-    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_tcgen05_launches", "cobs_sparse_decode_static",
+    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_tcgen05_launches", "cobs_sparse_decode_static", "cobs_append_token",
 ]
 
 
@@ -167,6 +167,15 @@ def cobs_build_summaries(cfg: Config, kv: KV, block_begin: int, block_end: int, 
     _check(lib().cobs_build_summaries(C.byref(cfg), C.byref(kv), C.c_int32(block_begin), C.c_int32(block_end),
                                       C.byref(s), _ptr(ws), C.c_size_t(ws.numel()), _stream(stream)),
            "cobs_build_summaries")
+
+
+def cobs_append_token(cfg: Config, k_new: torch.Tensor, v_new: torch.Tensor, inputs, ws: torch.Tensor, stream=None):
+    """Write one new token per sequence into the paged cache of `inputs` (k_pages, v_pages, page_table, seq_lens)
+    and advance seq_lens on the device."""
+    _check(lib().cobs_append_token(C.byref(cfg), _ptr(k_new), _ptr(v_new), _ptr(inputs["k_pages"]), _ptr(inputs["v_pages"]),
+                                   _ptr(inputs["page_table"]), _ptr(inputs["seq_lens"]),
+                                   C.c_int64(inputs["k_pages"].shape[0]), _ptr(ws), C.c_size_t(ws.numel()),
+                                   _stream(stream)), "cobs_append_token")
 
 
 def cobs_quantise_xi(cfg: Config, xi_fp32: torch.Tensor, codes: torch.Tensor, scale: torch.Tensor, stream=None):

@@ -18,6 +18,8 @@ cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream);
 bool fused_score_supported(const Params &p);
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
 cudaError_t launch_build(const Params &p, int block_begin, int block_end, cudaStream_t stream);
+cudaError_t launch_append(const Params &p, const void *k_new, const void *v_new, void *k_pages, void *v_pages, int32_t *seq_lens,
+                          int32_t *old_lens, cudaStream_t stream);
 cudaError_t launch_quantise(const float *xi, long long n_vectors, int Ds, int Ds_pad, int scale_dtype, void *codes,
                             void *scale, cudaStream_t stream);
 size_t build_smem_bytes(const Params &p);
@@ -259,6 +261,24 @@ int32_t cobs_build_summaries(const cobs_config *cfg, const cobs_kv *kv, int32_t 
   if ((st = set_summaries(p, cfg, out)) != COBS_OK) return st;
   if (build_smem_bytes(p) > 227 * 1024) return COBS_ERR_UNSUPPORTED;
   return cuda_status(launch_build(p, block_begin, block_end, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t cobs_append_token(const cobs_config *cfg, const void *k_new, const void *v_new, void *k_pages, void *v_pages,
+                          const int32_t *page_table, int32_t *seq_lens, int64_t n_pages, void *workspace,
+                          size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (!k_new || !v_new || !k_pages || !v_pages || !page_table || !seq_lens || n_pages < 1) return COBS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(k_pages) |
+       reinterpret_cast<uintptr_t>(v_pages)) % 16 != 0) return COBS_ERR_INVALID_ARG;
+  Params p;
+  fill_params(p, cfg, workspace);
+  p.page_table = page_table;
+  p.n_pages = n_pages;
+  // the snapshot of the lengths lives in the query staging area of the workspace (batch * 4 bytes of it)
+  int32_t *old_lens = reinterpret_cast<int32_t *>(static_cast<unsigned char *>(workspace) + layout_workspace(cfg).q_stage);
+  return cuda_status(launch_append(p, k_new, v_new, k_pages, v_pages, seq_lens, old_lens, static_cast<cudaStream_t>(stream)));
 }
 
 int32_t cobs_quantise_xi(const cobs_config *cfg, const float *xi_fp32, int64_t n_vectors, void *codes, void *scale,

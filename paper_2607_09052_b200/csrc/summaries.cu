@@ -338,6 +338,36 @@ cudaError_t launch_build(const Params &p, int block_begin, int block_end, cudaSt
   return cudaGetLastError();
 }
 
+// One new token per sequence into the paged cache: 16 bytes per thread, one CTA per (sequence, KV head); the
+// CTAs of KV head 0 also advance the sequence lengths once every CTA of the sequence has read the old one.
+__global__ void append_kernel(Params p, const __nv_bfloat16 *k_new, const __nv_bfloat16 *v_new, __nv_bfloat16 *k_pages,
+                              __nv_bfloat16 *v_pages, int32_t *seq_lens, const int32_t *old_lens) {
+  const int b = blockIdx.x / p.Hkv, h = blockIdx.x - b * p.Hkv;
+  const int T = old_lens[b];
+  if (T < 0 || T >= p.mpp * p.P) { if (threadIdx.x == 0) report(p.status, COBS_ERR_BOUNDS); return; }
+  const int pg = p.page_table[(size_t)b * p.mpp + T / p.P];
+  if (pg < 0 || pg >= p.n_pages) { if (threadIdx.x == 0) report(p.status, COBS_ERR_BOUNDS); return; }
+  const size_t dst = (((size_t)pg * p.Hkv + h) * p.P + (T % p.P)) * p.D, src = ((size_t)b * p.Hkv + h) * p.D;
+  for (int i = threadIdx.x; i < p.D / 8; i += blockDim.x) {
+    reinterpret_cast<uint4 *>(k_pages + dst)[i] = reinterpret_cast<const uint4 *>(k_new + src)[i];
+    reinterpret_cast<uint4 *>(v_pages + dst)[i] = reinterpret_cast<const uint4 *>(v_new + src)[i];
+  }
+  if (h == 0 && threadIdx.x == 0) seq_lens[b] = T + 1;
+}
+
+// old_lens: a snapshot of the lengths taken on the stream before the launch (the kernel reads the snapshot and
+// writes the live array, so no CTA can see a length another CTA has already advanced).
+cudaError_t launch_append(const Params &p, const void *k_new, const void *v_new, void *k_pages, void *v_pages, int32_t *seq_lens,
+                          int32_t *old_lens, cudaStream_t stream) {
+  cudaError_t e = cudaMemcpyAsync(old_lens, seq_lens, sizeof(int32_t) * p.B, cudaMemcpyDeviceToDevice, stream);
+  if (e != cudaSuccess) return e;
+  append_kernel<<<p.B * p.Hkv, 32, 0, stream>>>(p, static_cast<const __nv_bfloat16 *>(k_new), static_cast<const __nv_bfloat16 *>(v_new),
+                                                 static_cast<__nv_bfloat16 *>(k_pages), static_cast<__nv_bfloat16 *>(v_pages), seq_lens,
+                                                 old_lens);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_quantise(const float *xi, long long n_vectors, int Ds, int Ds_pad, int scale_dtype, void *codes,
                             void *scale, cudaStream_t stream) {
   if (n_vectors <= 0) return cudaSuccess;
