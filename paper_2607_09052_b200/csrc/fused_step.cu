@@ -3,23 +3,25 @@
 //
 // Why one kernel.  A step moves a few hundred MiB; at HBM speed that is tens of microseconds, so
 // every kernel boundary (launch, ramp-up, tail, the idle time while a single CTA per unit selects)
-// costs a visible fraction of the step.  Here the grid is sized to be fully resident (2 CTAs of 4
-// warps per SM) and every WARP runs the same program on its own share of the work:
+// costs a visible fraction of the step.  Here the grid is one CTA per SM, fully resident (cooperative
+// launch), with two kinds of warps:
 //
-//   phase S  score 16-block chunks of summaries (chunks dealt round-robin to all warps of the grid,
-//            so the grid sweeps the summary arrays front to back and units finish in order);
-//            the warp that finishes the last chunk of a (sequence, KV head) unit selects its top-k;
-//   phase A  attend over (unit, split) items, dealt round-robin in unit order; a warp whose slice
-//            holds selected blocks waits (bounded) for that unit's selection, slices that hold only
-//            window blocks never wait; the warp that finishes the last slice of a unit merges the
-//            partials and writes the output.
+//   streaming warps (8 per CTA), each with its own slice of shared memory:
+//     phase S  score 16-block chunks of summaries: the units are scored in waves, and inside a wave every
+//              warp takes one contiguous range of chunks; per chunk it leaves t = exp(e - chunk max) per
+//              block and head, the chunk's (max, sum) pair, and counts the chunk on its unit;
+//     phase A  attend over (unit, slice) items drawn from one global counter in unit order; a warp whose
+//              slice holds selected blocks waits (bounded) for that unit's selection, slices that hold only
+//              window blocks never wait; the warp that finishes the last slice of a unit merges the
+//              partials and writes the output;
+//   a selection team (4 warps per CTA) that selects unit u (team of CTA u mod grid) as soon as all its
+//     chunks are counted, while the streaming warps carry on with the next wave.
 //
-// Data movement.  Every stream a warp consumes goes global -> shared with cp.async into a ring that
-// belongs to that warp alone (no CTA barrier anywhere in the loops) and ALL streams of a phase have
-// the same prefetch depth: a shallower stream would set the pace while the deeper ones only add
-// queueing delay.  Scoring: thread-private 16-byte slots (a lane copies exactly the fragments it will
-// feed to the tensor core), depth 1.  Attention: K and V of a 16-token group share a stage
-// (XOR-swizzled 16-byte chunks, read back with ldmatrix / ldmatrix.trans), depth 2.
+// Data movement.  Every stream a warp consumes goes global -> shared into a ring that belongs to that warp
+// alone (no CTA barrier anywhere in the loops).  Scoring: a chunk is three contiguous pieces of the summary
+// arrays, fetched by three bulk copies (cp.async.bulk, completion on an mbarrier) issued by one lane, two
+// stages.  Attention: K and V of a 16-token group share a stage of a three-stage cp.async ring (XOR-swizzled
+// 16-byte chunks, read back with ldmatrix / ldmatrix.trans).
 //
 // Arithmetic.  mma.sync m16n8k16 with fp32 accumulation throughout:
 //   scoring   rows = 16 block means, or factor i of 16 blocks; columns = the G query heads.  A thread
@@ -29,6 +31,7 @@
 //             (exact in f16), or an f16 high + low split of the fp32 subspace query.
 //   attention S^T = q K^T with the heads as rows (zero padded to 16) and 8 tokens as columns; the S
 //             accumulators are the A fragments of P V as they sit in registers; P = bf16 high + low.
+// An opt-in variant runs phase S of the main configuration on tcgen05 (further down).
 //
 // Cross-warp hand-offs go through global counters in the workspace (release: write, __threadfence,
 // atomicAdd; acquire: volatile read, __threadfence, .cg loads).  Every wait is bounded; on expiry the
@@ -65,9 +68,6 @@ enum { PH_SCORE = 1, PH_ATTEND = 2 };
 #define COBS_WAVES 4
 #endif
 constexpr int kWaves = COBS_WAVES;                           // the units are scored in this many waves
-#ifndef COBS_EVEN_SHARES
-#define COBS_EVEN_SHARES 0                                   // scoring: equal chunk counts per warp instead of ceil-sized ranges
-#endif
 #ifndef COBS_SCORE_RG
 #define COBS_SCORE_RG 4                                      // FP4 factor rows decoded and multiplied together
 #endif
@@ -76,7 +76,6 @@ constexpr int kWaves = COBS_WAVES;                           // the units are sc
 // development aid: per-warp phase boundary timestamps (ns), read back by cobs_debug_times
 __device__ unsigned long long g_dbg_times[4][4096];
 __device__ unsigned long long g_dbg_acc[8][4096];   // per-warp accumulated clock cycles by category
-__device__ unsigned long long g_dbg_trace[32][64];  // event times of every 37th streaming warp
 __device__ __forceinline__ unsigned long long gtime() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -84,17 +83,11 @@ __device__ __forceinline__ unsigned long long gtime() {
 }
 #define COBS_STAMP(k) do { if (lane == 0 && wg < 4096) g_dbg_times[k][wg] = gtime(); } while (0)
 #define COBS_SEL_STAMP(k) do { if (tid == 0 && u < 1024) g_dbg_acc[k][3000 + u] = gtime(); } while (0)
-#define COBS_TRACE_DECL int trace_n = 0
-#define COBS_TRACE() do { if (lane == 0 && wg % 37 == 0 && trace_n < 64) g_dbg_trace[wg / 37][trace_n++] = gtime(); } while (0)
-#define COBS_TRACE1() do { if (first_chunk) COBS_TRACE(); } while (0)
 #define COBS_ACC_DECL long long acc_t[8] = {0,0,0,0,0,0,0,0}; long long acc_last = clock64()
 #define COBS_ACC(k) do { long long now_ = clock64(); acc_t[k] += now_ - acc_last; acc_last = now_; } while (0)
 #define COBS_ACC_FLUSH(id) do { if ((threadIdx.x & 31) == 0 && (id) < 4096) { for (int k_ = 0; k_ < 8; ++k_) g_dbg_acc[k_][id] += acc_t[k_]; } } while (0)
 #else
 #define COBS_ACC_DECL do { } while (0)
-#define COBS_TRACE_DECL do { } while (0)
-#define COBS_TRACE() do { } while (0)
-#define COBS_TRACE1() do { } while (0)
 #define COBS_ACC(k) do { } while (0)
 #define COBS_ACC_FLUSH(id) do { } while (0)
 #define COBS_STAMP(k) do { } while (0)
@@ -503,17 +496,12 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   auto wave_range = [&](int w, int &cb, int &ce) {          // this warp's chunk range [cb, ce) in wave w
     const int u0 = (units * w) / n_waves, u1 = (units * (w + 1)) / n_waves;
     const int tot = (u1 - u0) * cpu;                       // the host refuses configurations where this overflows
-#if COBS_EVEN_SHARES
-    // even shares (they differ by at most one chunk); the warps that get the larger share rotate with the wave
-    int wr = wg + w * (n_wg / n_waves + 1);
-    wr -= (wr / n_wg) * n_wg;
-    cb = u0 * cpu + (int)(((long long)wr * tot) / n_wg);
-    ce = u0 * cpu + (int)(((long long)(wr + 1) * tot) / n_wg);
-#else
+    // ceil-sized ranges: at the benchmark's size this leaves the last 20 CTAs without scoring work; they start on the
+    // attention of the first selected units while the others still score, which measured 5 us faster per step than
+    // equal shares for every warp
     const int per = (tot + n_wg - 1) / n_wg;
     cb = u0 * cpu + min(wg * per, tot);
     ce = u0 * cpu + min(wg * per + per, tot);
-#endif
   };
   // first position at or after (u, ck) that holds work, moving on to the next wave's range when this one is
   // exhausted; u = units when there is nothing left.  Chunk 0 of a unit without summarised blocks counts as work:
@@ -534,8 +522,6 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   };
 
   COBS_ACC_DECL;
-  COBS_TRACE_DECL;
-  COBS_TRACE();
   // ---- bulk copies of (chunk c, batch b) into stage st; completion is counted on the stage's mbarrier ----
   // lanes 0-15 copy the factor rows of block `lane`, lanes 16-31 the mean of block `lane - 16`, lane 0 the scales
   auto issue = [&](int u, int ck, int n_sum, int b, int st) {
@@ -609,9 +595,6 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   int cur_u = -1;
   bool alive = true;
 
-  bool first_chunk = true;
-  (void)first_chunk;
-  COBS_TRACE();
   while (cu < units && alive) {
     COBS_ACC(0);
     // ---- prefetch the next batch of this warp --------------------------------------------------------
@@ -624,7 +607,6 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     COBS_ACC(6);
     issue(nu, nck, nn, nxt_b, st ^ 1);
     COBS_ACC(1);
-    COBS_TRACE1();
 
     const int u = cu, ck = cck, n_sum = cn;
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
@@ -638,8 +620,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
       phase_bits ^= 1u << st;
       __syncwarp();
       COBS_ACC(2);
-      COBS_TRACE1();
-      if (cur_b == 0) {
+        if (cur_b == 0) {
         if (u != cur_u) {
           cur_u = u;
           // ---- query fragments of this unit ------------------------------------------------------------
@@ -699,8 +680,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
             m1 = __shfl_sync(0xffffffffu, mult, (2 * tig + 1) * 4);
           }
         }
-        COBS_TRACE1();
-        // ---- first-order term: block means against the raw bf16 query ------------------------------------
+            // ---- first-order term: block means against the raw bf16 query ------------------------------------
         float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;   // two chains
         const uint32_t ma = sbase + (2 * gid) * mrow + tig * 16, mb = ma + mrow;
 #pragma unroll
@@ -798,8 +778,6 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     }
 
     COBS_ACC(3);
-    COBS_TRACE1();
-    first_chunk = false;
     // ---- end of a chunk: publish t = exp(e - chunk max) per block and the chunk's (max, sum of t) per head ----
     if (cur_b == n_batches - 1) {
       if (pend_u != u && pend_n > 0) {       // moving on to another unit: count the finished one's chunks
@@ -848,7 +826,6 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     }
     __syncwarp();                           // all lanes are done with stage st before it is refilled
     COBS_ACC(4);
-    COBS_TRACE();
     cu = nu; cck = nck; cn = nn; cur_b = nxt_b; st ^= 1;
   }
   if (pend_n > 0) {
@@ -1614,13 +1591,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
     }
     __syncwarp();
     COBS_STAMP(0);
-#ifdef COBS_SCORE_WARPS
-    if ((phases & PH_SCORE) && warp < COBS_SCORE_WARPS)
-      score_phase<DT, D, WPT, NT>(p, seq_lens, wsm, &s_bars[warp][0], blockIdx.x * COBS_SCORE_WARPS + warp,
-                                  gridDim.x * COBS_SCORE_WARPS, lane);
-#else
     if (phases & PH_SCORE) score_phase<DT, D, WPT, NT>(p, seq_lens, wsm, &s_bars[warp][0], wg, n_wg, lane);
-#endif
     COBS_STAMP(1);
     COBS_STAMP(2);
     if (phases & PH_ATTEND) attend_phase<D>(p, seq_lens, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
@@ -1936,12 +1907,6 @@ extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void 
 #ifdef COBS_TIMING
 extern "C" int cobs_debug_times(unsigned long long *host_out) {
   return (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_times, sizeof(unsigned long long) * 4 * 4096);
-}
-extern "C" int cobs_debug_trace(unsigned long long *host_out) {
-  int e = (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_trace, sizeof(unsigned long long) * 32 * 64);
-  static unsigned long long z[32 * 64];
-  cudaMemcpyToSymbol(cobs::g_dbg_trace, z, sizeof(z));
-  return e;
 }
 extern "C" int cobs_debug_acc(unsigned long long *host_out, int clear) {
   int e = (int)cudaMemcpyFromSymbol(host_out, cobs::g_dbg_acc, sizeof(unsigned long long) * 8 * 4096);
