@@ -3,8 +3,12 @@
 //   mean   = (1/L) sum_t k_t                                  (Eq. cgf-cumulants)
 //   K~     = rows k_t - mean  (times U_Q for the subspace descriptor)
 //   C      = K~ K~^T / L      (L x L Gram matrix)             (Method, Cost: Gram trick)
-//   (lambda_i, w_i) = eigenpairs of C by parallel cyclic Jacobi, lambda descending
+//   (lambda_i, w_i) = eigenpairs of C, lambda descending
 //   xi_i   = K~^T w_i / sqrt(L)  = sqrt(lambda_i) u_i         (Eq. lowrank)
+// computed without forming C: one-sided (Hestenes) Jacobi rotates pairs of ROWS of K~ until all rows are mutually
+// orthogonal.  The product of the rotations is W^T, so the rows end up as K~^T w_i = sqrt(L) xi_i with squared
+// norms L lambda_i: the same O(L^2 D) work per sweep as the Gram route, the L x L matrices never exist, and a
+// rotation is one dot product and one update of two rows held by a warp.
 //   store  : fp32 | bf16 (RNE) | FP4 E2M1 + one scale per factor (Method, Quantization)
 //
 // One CTA per (sequence, KV head, block); everything stays in shared memory.  All reductions run in
@@ -15,6 +19,10 @@ namespace cobs {
 
 constexpr int kBuildThreads = 256;
 constexpr int kMaxSweeps = 16;
+
+// row stride of the centred keys in shared memory: a multiple of 4 floats (rows are read 16 bytes per lane), plus
+// 4 so that consecutive rows start in different banks
+__host__ __device__ inline int build_ldk(const Params &p) { return (((p.D > p.Ds) ? p.D : p.Ds) + 3) / 4 * 4 + 4; }
 
 // --- FP4 quantiser -------------------------------------------------------------------------------
 // code = sign bit of x, nearest E2M1 magnitude to |x| / scale with ties to the even mantissa bit.
@@ -73,16 +81,13 @@ __global__ void quantise_kernel(const float *xi, long long n_vectors, int Ds, in
 //                 small arrays
 __global__ void __launch_bounds__(kBuildThreads) build_kernel(Params p, int block_begin, int block_end) {
   extern __shared__ __align__(16) float sm[];
-  const int L = p.L, D = p.D, Dk = p.Ds, ldk = ((D > Dk) ? D : Dk) + 1, ldc = L + 1;
-  float *Kc = sm;                        // [L][ldk]
-  float *C = Kc + L * ldk;               // [L][ldc]
-  float *W = C + L * ldc;                // [L][ldc]
-  float *rot_c = W + L * ldc;            // [L / 2]
-  float *rot_s = rot_c + L / 2;          // [L / 2]
-  float *vec = rot_s + L / 2;            // [max(D, L)] scratch: mean, then eigenvalues
-  float *red = vec + ((D > L) ? D : L);  // [2 * kBuildThreads / 32]
-  float *wnorm = red + 2 * (kBuildThreads / 32);                      // [r] 1 / |w_i|
-  int *top = reinterpret_cast<int *>(wnorm + COBS_MAX_RANK);          // [r]
+  const int L = p.L, D = p.D, Dk = p.Ds, ldk = build_ldk(p);
+  float *Kc = sm;                        // [L][ldk] centred keys; rotated in place into sqrt(L) xi rows
+  float *nrm = Kc + L * ldk;             // [L] squared row norms
+  float *vec = nrm + L;                  // [max(D, L)] scratch: mean, then eigenvalues
+  float *red = vec + ((D > L) ? D : L);  // [kBuildThreads / 32]
+  int *top = reinterpret_cast<int *>(red + kBuildThreads / 32);       // [r]
+  int *flag = top + COBS_MAX_RANK;                                     // [1] a rotation was applied in this sweep
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int NW = kBuildThreads / 32;
@@ -148,101 +153,104 @@ __global__ void __launch_bounds__(kBuildThreads) build_kernel(Params p, int bloc
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int s = lane + 32 * i;
-        if (s < Dk) Kc[t * ldk + s] = o[i];
+        if (s < D) Kc[t * ldk + s] = (s < Dk) ? o[i] : 0.f;        // columns past the subspace are cleared
       }
     }
     __syncthreads();
   }
 
-  // ---- Gram matrix C = K~ K~^T / L,  W = I ---------------------------------------------------------
-  const float inv_l = 1.0f / (float)L;
-  for (int c = tid; c < L * L; c += kBuildThreads) {
-    const int i = c / L, j = c - i * L;
-    if (j >= i) {
-      float s = 0.f;
-      for (int d = 0; d < Dk; ++d) s = fmaf(Kc[i * ldk + d], Kc[j * ldk + d], s);
-      s *= inv_l;
-      C[i * ldc + j] = s;
-      C[j * ldc + i] = s;
-    }
-    W[i * ldc + j] = (i == j) ? 1.f : 0.f;
-  }
-  __syncthreads();
-
-  // ---- parallel cyclic Jacobi (round-robin pairing), two-sided on C, rotations accumulated in W ----
-  const int half = L / 2;
-  float prev_off = INFINITY;
+  // ---- one-sided Jacobi on the rows of K~ (round-robin pairing: L / 2 disjoint pairs per round) --------
+  // A half-warp owns a pair: lane l (of 16) holds columns 4 l .. 4 l + 3 and 64 + 4 l .. 64 + 4 l + 3 of both rows.
+  // Pair slot s of round R joins rows (R + s) mod (L - 1) and (R - s) mod (L - 1); slot 0 joins row L - 1 and row R.
+  const int half = L / 2, Dk4 = (Dk + 3) / 4 * 4;
+  const int hw = lane >> 4, l16 = lane & 15;
+  const bool col0 = 4 * l16 < Dk4, col1 = 64 + 4 * l16 < Dk4;
+  constexpr int NI = 4;                                   // pair slots per half-warp per round (L <= 128)
   for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
-    // convergence: off-diagonal mass against diagonal mass (every thread computes the same totals)
-    float off = 0.f, dia = 0.f;
-    for (int c = tid; c < L * L; c += kBuildThreads) {
-      const int i = c / L, j = c - i * L;
-      const float x = C[i * ldc + j];
-      if (i == j) dia = fmaf(x, x, dia); else off = fmaf(x, x, off);
+    // exact squared norms at the start of every sweep (they are updated by formula inside it)
+    for (int t = warp; t < L; t += NW) {
+      float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (4 * lane < Dk4) x = *reinterpret_cast<const float4 *>(Kc + t * ldk + 4 * lane);
+      const float s = warp_sum(fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, x.w * x.w))));
+      if (lane == 0) nrm[t] = s;
     }
-    off = warp_sum(off); dia = warp_sum(dia);
+    if (tid == 0) *flag = 0;
     __syncthreads();
-    if (lane == 0) { red[warp] = off; red[NW + warp] = dia; }
-    __syncthreads();
-    float off_t = 0.f, dia_t = 0.f;
-    for (int w = 0; w < NW; ++w) { off_t += red[w]; dia_t += red[NW + w]; }
-    // done when the off-diagonal mass is at rounding level, or small and no longer shrinking
-    if (off_t <= 1e-13f * dia_t || dia_t == 0.f) break;
-    if (off_t <= 1e-10f * dia_t && off_t > 0.5f * prev_off) break;
-    prev_off = off_t;
-
+    float nmax = 0.f;
+    for (int t = 0; t < L; ++t) nmax = fmaxf(nmax, nrm[t]);
+    const float floor2 = 1e-20f * nmax * nmax;            // rows below 1e-10 of the largest norm count as zero
+    int pi_[NI], qi_[NI];                                 // this half-warp's pairs, advanced round by round
+#pragma unroll
+    for (int j = 0; j < NI; ++j) {
+      const int slot = 2 * warp + hw + 2 * NW * j;
+      pi_[j] = (slot == 0) ? L - 1 : slot;
+      qi_[j] = (slot == 0) ? 0 : L - 1 - slot;
+    }
     for (int round = 0; round < L - 1; ++round) {
-      if (tid < half) {
-        int pi, qi;
-        if (tid == 0) { pi = L - 1; qi = round; }
-        else { pi = (round + tid) % (L - 1); qi = (round - tid + (L - 1)) % (L - 1); }
-        if (pi > qi) { const int t = pi; pi = qi; qi = t; }
-        const float app = C[pi * ldc + pi], aqq = C[qi * ldc + qi], apq = C[pi * ldc + qi];
-        float cs = 1.f, sn = 0.f;
-        if (fabsf(apq) > 1e-30f && fabsf(apq) > 1e-9f * sqrtf(fabsf(app * aqq))) {
-          const float theta = (aqq - app) / (2.f * apq);
-          const float tt = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(fmaf(theta, theta, 1.f)));
-          cs = rsqrtf(fmaf(tt, tt, 1.f));
-          sn = tt * cs;
+#pragma unroll
+      for (int j = 0; j < NI; ++j) {
+        if (2 * NW * j >= half) break;                      // no slot of this index in a round (uniform)
+        const int slot = 2 * warp + hw + 2 * NW * j;
+        const bool on = slot < half;
+        const int pi = on ? min(pi_[j], qi_[j]) : 0, qi = on ? max(pi_[j], qi_[j]) : 0;
+        float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1 = x0, y0 = x0, y1 = x0;
+        if (on && col0) {
+          x0 = *reinterpret_cast<const float4 *>(Kc + pi * ldk + 4 * l16);
+          y0 = *reinterpret_cast<const float4 *>(Kc + qi * ldk + 4 * l16);
         }
-        rot_c[tid] = cs; rot_s[tid] = sn;
-      }
-      __syncthreads();
-      // rows: C <- J^T C
-      for (int c = tid; c < half * L; c += kBuildThreads) {
-        const int pr = c / L, j = c - pr * L;
-        int pi, qi;
-        if (pr == 0) { pi = L - 1; qi = round; }
-        else { pi = (round + pr) % (L - 1); qi = (round - pr + (L - 1)) % (L - 1); }
-        if (pi > qi) { const int t = pi; pi = qi; qi = t; }
-        const float cs = rot_c[pr], sn = rot_s[pr];
-        const float x = C[pi * ldc + j], y = C[qi * ldc + j];
-        C[pi * ldc + j] = cs * x - sn * y;
-        C[qi * ldc + j] = sn * x + cs * y;
-      }
-      __syncthreads();
-      // columns: C <- C J,  W <- W J
-      for (int c = tid; c < half * L; c += kBuildThreads) {
-        const int pr = c / L, j = c - pr * L;
-        int pi, qi;
-        if (pr == 0) { pi = L - 1; qi = round; }
-        else { pi = (round + pr) % (L - 1); qi = (round - pr + (L - 1)) % (L - 1); }
-        if (pi > qi) { const int t = pi; pi = qi; qi = t; }
-        const float cs = rot_c[pr], sn = rot_s[pr];
-        float x = C[j * ldc + pi], y = C[j * ldc + qi];
-        C[j * ldc + pi] = cs * x - sn * y;
-        C[j * ldc + qi] = sn * x + cs * y;
-        x = W[j * ldc + pi]; y = W[j * ldc + qi];
-        W[j * ldc + pi] = cs * x - sn * y;
-        W[j * ldc + qi] = sn * x + cs * y;
+        if (on && col1) {
+          x1 = *reinterpret_cast<const float4 *>(Kc + pi * ldk + 64 + 4 * l16);
+          y1 = *reinterpret_cast<const float4 *>(Kc + qi * ldk + 64 + 4 * l16);
+        }
+        float g = fmaf(x0.x, y0.x, fmaf(x0.y, y0.y, fmaf(x0.z, y0.z, x0.w * y0.w))) +
+                  fmaf(x1.x, y1.x, fmaf(x1.y, y1.y, fmaf(x1.z, y1.z, x1.w * y1.w)));
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
+        const float a = nrm[pi], b = nrm[qi];
+        __syncwarp();
+        // rotate unless the rows are orthogonal to 4e-6 (the dot product of D terms is itself only good to ~1e-6)
+        if (on && a * b > floor2 && g * g > 1.6e-11f * (a * b)) {
+          // the angle may be approximate (any near-optimal rotation converges); c and s must satisfy
+          // c^2 + s^2 = 1 to an unbiased rounding, or the row norms drift: c comes from a correctly rounded rsqrt
+          const float zeta = __fdividef(b - a, 2.f * g);
+          const float az = fabsf(zeta), rt = (az < 1e18f) ? sqrtf(fmaf(zeta, zeta, 1.f)) : az;
+          const float tt = copysignf(__fdividef(1.f, az + rt), zeta);
+          const float cs = __frsqrt_rn(fmaf(tt, tt, 1.f)), sn = tt * cs;
+          if (col0) {
+            *reinterpret_cast<float4 *>(Kc + pi * ldk + 4 * l16) =
+                make_float4(cs * x0.x - sn * y0.x, cs * x0.y - sn * y0.y, cs * x0.z - sn * y0.z, cs * x0.w - sn * y0.w);
+            *reinterpret_cast<float4 *>(Kc + qi * ldk + 4 * l16) =
+                make_float4(sn * x0.x + cs * y0.x, sn * x0.y + cs * y0.y, sn * x0.z + cs * y0.z, sn * x0.w + cs * y0.w);
+          }
+          if (col1) {
+            *reinterpret_cast<float4 *>(Kc + pi * ldk + 64 + 4 * l16) =
+                make_float4(cs * x1.x - sn * y1.x, cs * x1.y - sn * y1.y, cs * x1.z - sn * y1.z, cs * x1.w - sn * y1.w);
+            *reinterpret_cast<float4 *>(Kc + qi * ldk + 64 + 4 * l16) =
+                make_float4(sn * x1.x + cs * y1.x, sn * x1.y + cs * y1.y, sn * x1.z + cs * y1.z, sn * x1.w + cs * y1.w);
+          }
+          if (l16 == 0) { nrm[pi] = fmaxf(a - tt * g, 0.f); nrm[qi] = b + tt * g; *flag = 1; }
+        }
+        // next round's rows of this slot
+        if (slot == 0) { qi_[j] = round + 1; }
+        else {
+          pi_[j] = (pi_[j] + 1 == L - 1) ? 0 : pi_[j] + 1;
+          qi_[j] = (qi_[j] + 1 == L - 1) ? 0 : qi_[j] + 1;
+        }
       }
       __syncthreads();
     }
+    if (*flag == 0) break;
+    __syncthreads();
   }
   __syncthreads();
 
-  // ---- top-r eigenvalues (descending, lower index on ties), by warp 0 ------------------------------
-  if (tid < L) vec[tid] = C[tid * ldc + tid];
+  // ---- eigenvalues = squared row norms / L; the top r (descending, lower index on ties), by warp 0 -----
+  for (int t = warp; t < L; t += NW) {
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (4 * lane < Dk4) x = *reinterpret_cast<const float4 *>(Kc + t * ldk + 4 * lane);
+    const float s = warp_sum(fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, x.w * x.w))));
+    if (lane == 0) vec[t] = s / (float)L;
+  }
   __syncthreads();
   if (warp == 0) {
     for (int i = 0; i < p.r; ++i) {
@@ -265,27 +273,13 @@ __global__ void __launch_bounds__(kBuildThreads) build_kernel(Params p, int bloc
   }
   __syncthreads();
 
-  // ---- rotations in fp32 are orthogonal only to rounding: renormalise the chosen eigenvectors ------
-  for (int i = warp; i < p.r; i += NW) {
-    const int col = top[i];
-    float s = 0.f;
-    if (col >= 0)
-      for (int t = lane; t < L; t += 32) s = fmaf(W[t * ldc + col], W[t * ldc + col], s);
-    s = warp_sum(s);
-    if (lane == 0) wnorm[i] = (col >= 0 && s > 0.f) ? 1.0f / sqrtf(s) : 0.f;
-  }
-  __syncthreads();
-
-  // ---- factors xi_i = K~^T w_i / sqrt(L), written over C (its diagonal has been copied out) -----------
-  float *xi_s = C;   // [r][Dk]
+  // ---- factors xi_i = (rotated row) / sqrt(L), gathered into the first rows' place holder ----------------
+  float *xi_s = nrm + L + ((D > L) ? D : L) + kBuildThreads / 32 + 2 * COBS_MAX_RANK;   // [r][Dk] after the small arrays
   const float inv_sqrt_l = 1.0f / sqrtf((float)L);
   for (int c = tid; c < p.r * Dk; c += kBuildThreads) {
     const int i = c / Dk, d = c - i * Dk;
     const int col = top[i];
-    float s = 0.f;
-    if (col >= 0)
-      for (int t = 0; t < L; ++t) s = fmaf(Kc[t * ldk + d], W[t * ldc + col], s);
-    xi_s[c] = (col >= 0) ? s * wnorm[i] * inv_sqrt_l : 0.f;
+    xi_s[c] = (col >= 0) ? Kc[col * ldk + d] * inv_sqrt_l : 0.f;
   }
   __syncthreads();
 
@@ -320,10 +314,10 @@ __global__ void __launch_bounds__(kBuildThreads) build_kernel(Params p, int bloc
 }
 
 size_t build_smem_bytes(const Params &p) {
-  const int L = p.L, ldk = ((p.D > p.Ds) ? p.D : p.Ds) + 1, ldc = L + 1;
-  size_t f = (size_t)L * ldk + 2 * (size_t)L * ldc + L + ((p.D > L) ? p.D : L) + 2 * (kBuildThreads / 32) +
-             COBS_MAX_RANK;
-  return f * sizeof(float) + (size_t)(COBS_MAX_RANK + 1) * sizeof(int);
+  const int L = p.L;
+  size_t f = (size_t)L * build_ldk(p) + L + ((p.D > L) ? p.D : L) + kBuildThreads / 32 + 2 * COBS_MAX_RANK +
+             (size_t)COBS_MAX_RANK * p.Ds;
+  return f * sizeof(float);
 }
 
 cudaError_t launch_build(const Params &p, int block_begin, int block_end, cudaStream_t stream) {
