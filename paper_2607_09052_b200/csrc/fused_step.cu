@@ -702,7 +702,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
         // RG factor rows at a time: RG independent accumulator chains keep the tensor pipe busy
         constexpr int RG = COBS_SCORE_RG;
         const unsigned char *sp = wsm + st * kScoreStageBytes + (kScoreStageBytes - scale_bytes) + (2 * gid) * r * scale_sz;
-#pragma unroll
+#pragma unroll 1
         for (int i0 = 0; i0 < ROWS_MAX; i0 += RG) {
           if (i0 < rows) {
             float d[RG][4];
