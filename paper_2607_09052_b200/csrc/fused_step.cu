@@ -491,7 +491,9 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   // scored - or, for the last wave, while the first wave's units are being attended.
   // A position is (unit, chunk-in-unit, blocks of the unit); 32-bit arithmetic throughout.
   auto unit_blocks = [&](int u) -> int { return min(seq_lens[u / p.Hkv] / L, NB); };
-  const int n_waves = (units >= 2 * kWaves) ? kWaves : 1;
+  // waves only when there is enough work to keep every warp busy in each of them: with fewer chunks than warps a
+  // wave would serialise chunks on a few warps while the rest idle
+  const int n_waves = max(1, min(min(kWaves, units / 2), (units * cpu) / n_wg));
   int wave = 0, c_end = 0;
   auto wave_range = [&](int w, int &cb, int &ce) {          // this warp's chunk range [cb, ce) in wave w
     const int u0 = (units * w) / n_waves, u1 = (units * (w + 1)) / n_waves;
