@@ -74,10 +74,15 @@ static int32_t validate_config(const cobs_config *c) {
 static int choose_splits(const cobs_config *c) {
   const int units = c->batch * c->n_kv_heads;
   const int groups = max_items(c) * (c->block_size / 16);
-#ifndef COBS_ITEMS_PER_WARP
-#define COBS_ITEMS_PER_WARP 2
+  // Two slices per streaming warp when the scoring runs in waves (then the second round of items absorbs the units
+  // whose selection finishes last); one per warp otherwise (an item costs several microseconds beyond its bytes).
+  const long long chunks = (long long)units * ((c->max_blocks + 15) / 16);
+#ifdef COBS_ITEMS_PER_WARP
+  const int per_warp = COBS_ITEMS_PER_WARP;
+#else
+  const int per_warp = (chunks / kGridWarps >= 2) ? 2 : 1;
 #endif
-  int s = COBS_ITEMS_PER_WARP * kGridWarps / units;   // a few slices per streaming warp: the item queue balances them
+  int s = per_warp * kGridWarps / units;
   const int need = (groups + kItemGroups - 1) / kItemGroups;
   if (s < need) s = need;
   // small batches: more slices shorten each slice's stream (about 1.2 us per 16-token group) but lengthen the merge
