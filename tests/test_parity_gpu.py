@@ -195,6 +195,14 @@ def test_ragged_lengths_and_degenerate_cases():
     run_stage_s(wl)
 
 
+def test_context_beyond_the_fused_selection_capacity():
+    """4096 blocks per unit: more than the step kernel's selection team holds (2048), so scoring and selection
+    take the generic kernels and only attention runs in the persistent kernel; same parity bar."""
+    wl = synth.Workload("long", 1, 4, 1, 128, 4096 * 64, 64, 64, rank=4, topk=16, window=512, summary_dtype="fp4",
+                        key_model="block_offset", planted=4, shuffle_pages=False, seed=41)
+    run_stage_s(wl)
+
+
 def test_rank_zero_is_first_order_mean_pool():
     wl = WL["cfg1_tiny"].replace(rank=0, summary_dtype="bf16")
     run_stage_s(wl)
