@@ -176,7 +176,8 @@ def run_ours(args):
     t_warm = time.perf_counter()
     n_warm = 0
     while n_warm < args.warmup or time.perf_counter() - t_warm < args.clock_warm_s:   # >= W steps, and long enough for clock samples
-        flush.zero_()
+        if not args.no_l2_flush:
+            flush.zero_()
         step()
         n_warm += 1
         if n_warm % 16 == 0:
@@ -189,7 +190,8 @@ def run_ours(args):
     launches0 = B.cobs_kernel_launches()
     t_wall0 = time.perf_counter()
     for i in range(args.steps):
-        flush.zero_()
+        if not args.no_l2_flush:
+            flush.zero_()
         starts[i].record(stream)
         step()
         ends[i].record(stream)
@@ -288,7 +290,8 @@ def run_ours(args):
                    "page_size": wl.page_size, "topk": wl.topk, "window": wl.window, "rank": wl.rank,
                    "sub_dim": wl.sub_dim, "summary_dtype": wl.summary_dtype, "scale_dtype": wl.scale_dtype,
                    "record_bytes": record, "algorithmic_bytes_per_step": step_bytes,
-                   "l2": f"{L2_FLUSH_BYTES >> 20} MiB write between timed steps (outside the events); "
+                   "l2": ("no flush: " if args.no_l2_flush else
+                          f"{L2_FLUSH_BYTES >> 20} MiB write between timed steps (outside the events); ") +
                          f"step traffic {step_bytes / 2**20:.1f} MiB",
                    "sharding": "independent sequences per rank, no collective"},
         "frac_of_measured_peak": round(value / (world * peak), 4), "peak_gbs": peak, "peak_kind": peak_kind,
@@ -419,6 +422,8 @@ def main():
     ap.add_argument("--seq-len", type=int, default=0, help="override the workload's context (profiling on a small case)")
     ap.add_argument("--contiguous-pages", action="store_true",
                     help="diagnostic: identity page table instead of the workload's shuffled pages")
+    ap.add_argument("--no-l2-flush", action="store_true",
+                    help="do not write 256 MiB between timed steps (valid only where the step's own traffic exceeds L2)")
     ap.add_argument("--decode-loop", type=int, default=0,
                     help="also time this many consecutive decode steps (append, rebuild on block fill, step) and "
                          "report the amortised time per step")
