@@ -182,6 +182,17 @@ int32_t cobs_score_select(const cobs_config *cfg, const void *q, const cobs_summ
                           size_t workspace_bytes, void *stream);
 
 /*
+ * The exact-mass selector (the paper's oracle sparse attention, OSA; Eq. bg-defs, Eq. prop-gqa): as
+ * cobs_score_select, but every full block's log mass is the direct sum over its keys,
+ *   e[g][b] = ln sum_{t in b} exp(q'_g . k_t),
+ * instead of the second-order estimate from the summaries.  Same group score, candidates, tie rule and outputs.
+ * It reads every key of the cache (the work the estimator avoids): a quality reference, not a step of the
+ * decode path.  Reads cfg's shapes, block_size, page_size, topk, window, max_blocks only.
+ */
+int32_t cobs_exact_select(const cobs_config *cfg, const void *q, const cobs_kv *kv, int32_t *sel_idx, int32_t *sel_cnt,
+                          float *scores_or_null, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * (d) Attention over the selected blocks and the window, one softmax over their union
  * (Eq. oracle-true restricted to the kept blocks and the window).
  * out [B][Hq][D] fp32; lse_or_null [B][Hq] fp32 = log of the softmax denominator (natural log).

@@ -23,7 +23,7 @@ SCALE_DTYPES = {"fp32": 0, "fp16": 1}
 EXPORTS = [
     "cobs_status_string", "cobs_padded_sub_dim", "cobs_summary_bytes", "cobs_workspace_bytes", "cobs_reset_status",
     "cobs_read_status", "cobs_build_summaries", "cobs_quantise_xi", "cobs_score_select", "cobs_sparse_decode",
-    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_tcgen05_launches", "cobs_sparse_decode_static", "cobs_append_token",
+    "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_tcgen05_launches", "cobs_sparse_decode_static", "cobs_append_token", "cobs_exact_select",
 ]
 
 
@@ -191,6 +191,13 @@ def cobs_score_select(cfg: Config, q: torch.Tensor, summ: SummaryBuffers, seq_le
     _check(lib().cobs_score_select(C.byref(cfg), _ptr(q), C.byref(s), _ptr(seq_lens), _ptr(sel_idx), _ptr(sel_cnt),
                                    _ptr(scores), _ptr(ws), C.c_size_t(ws.numel()), _stream(stream)),
            "cobs_score_select")
+
+
+def cobs_exact_select(cfg: Config, q: torch.Tensor, kv: KV, sel_idx: torch.Tensor, sel_cnt: torch.Tensor,
+                      scores: Optional[torch.Tensor], ws: torch.Tensor, stream=None):
+    """Selection by exact block masses (reads every key): the quality reference for cobs_score_select."""
+    _check(lib().cobs_exact_select(C.byref(cfg), _ptr(q), C.byref(kv), _ptr(sel_idx), _ptr(sel_cnt), _ptr(scores),
+                                   _ptr(ws), C.c_size_t(ws.numel()), _stream(stream)), "cobs_exact_select")
 
 
 def cobs_sparse_decode(cfg: Config, q: torch.Tensor, kv: KV, sel_idx: torch.Tensor, sel_cnt: torch.Tensor,

@@ -14,6 +14,7 @@ void count_tcgen05_launch() { g_tc_launches.fetch_add(1, std::memory_order_relax
 
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_select(const Params &p, cudaStream_t stream);
+cudaError_t launch_exact_mass(const Params &p, cudaStream_t stream);
 cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream);
 bool fused_score_supported(const Params &p);
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
@@ -324,6 +325,22 @@ int32_t cobs_score_select(const cobs_config *cfg, const void *q, const cobs_summ
   }
   cudaError_t e = launch_score(p, s);
   if (e != cudaSuccess) return COBS_ERR_CUDA;
+  return cuda_status(launch_select(p, s));
+}
+
+int32_t cobs_exact_select(const cobs_config *cfg, const void *q, const cobs_kv *kv, int32_t *sel_idx, int32_t *sel_cnt,
+                          float *scores_or_null, void *workspace, size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (!q || !aligned16(q) || !sel_idx || !sel_cnt) return COBS_ERR_INVALID_ARG;
+  Params p;
+  fill_params(p, cfg, workspace);
+  if ((st = set_kv(p, kv)) != COBS_OK) return st;
+  p.q = static_cast<const __nv_bfloat16 *>(q);
+  p.sel_idx = sel_idx; p.sel_cnt = sel_cnt; p.scores = scores_or_null;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (launch_exact_mass(p, s) != cudaSuccess) return COBS_ERR_CUDA;
   return cuda_status(launch_select(p, s));
 }
 

@@ -1,7 +1,8 @@
 """Variants of the descriptor on one shape, through the same kernels: rank 0 (mean-pool score), 4, 6, 8; full key
 space or a query subspace of several widths; bf16 or FP4 factors (the paper's ablation axes: Table "bandwidth",
 Table "quant", the per-layer subspace widths).  For every variant: the record bytes per block and KV head, the
-algorithmic bytes of a decode step, and the measured step time on the GPU.  Prints a markdown table.
+algorithmic bytes of a decode step, the measured step time on the GPU, and the recall of its selection against the
+exact-mass selector (cobs_exact_select, the paper's OSA reference).  Prints a markdown table.
 
     python -m paper_2607_09052_b200.sweep [--batch 4] [--steps 30]
 
@@ -62,7 +63,16 @@ def time_variant(wl: synth.Workload, steps: int):
     us = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)[len(evs) // 2]
     mb, xb, sb = B.cobs_summary_bytes(cfg)
     record = (mb + xb + sb) // (nb * hkv * wl.max_blocks)
-    return record, algorithmic_bytes(wl, record), us
+    # recall of the estimator's selection against the exact-mass selector (the paper's OSA reference)
+    sel_x, cnt_x = torch.zeros_like(sel), torch.zeros_like(cnt)
+    B.cobs_exact_select(cfg, inp["q"], kv, sel_x, cnt_x, None, ws)
+    torch.cuda.synchronize()
+    hits = total = 0
+    for a, b in zip(sel.cpu().reshape(-1, wl.topk).tolist(), sel_x.cpu().reshape(-1, wl.topk).tolist()):
+        want = {x for x in b if x >= 0}
+        hits += len(want & {x for x in a if x >= 0})
+        total += len(want)
+    return record, algorithmic_bytes(wl, record), us, hits / max(total, 1)
 
 
 def main():
@@ -83,11 +93,12 @@ def main():
     variants.append(("subspace s=85, r=4, bf16", base.replace(sub_dim=85, rank=4, summary_dtype="bf16")))
     print(f"shape: B={base.batch}, {base.n_q_heads} query / {base.n_kv_heads} KV heads, D={base.head_dim}, "
           f"T={base.seq_len}, L={base.block_size}, k={base.topk}, W={base.window}")
-    print("| descriptor | record B / block / KV head | algorithmic MiB / step | step (median, us) | GB/s |")
-    print("|---|---|---|---|---|")
+    print("| descriptor | record B / block / KV head | algorithmic MiB / step | step (median, us) | GB/s | "
+          "recall of the exact-mass top-k |")
+    print("|---|---|---|---|---|---|")
     for label, wl in variants:
-        record, nbytes, us = time_variant(wl.replace(name=label), args.steps)
-        print(f"| {label} | {record} | {nbytes / 2**20:.1f} | {us:.1f} | {nbytes / us / 1e3:.0f} |")
+        record, nbytes, us, recall = time_variant(wl.replace(name=label), args.steps)
+        print(f"| {label} | {record} | {nbytes / 2**20:.1f} | {us:.1f} | {nbytes / us / 1e3:.0f} | {recall:.3f} |")
 
 
 if __name__ == "__main__":

@@ -173,6 +173,46 @@ def test_tcgen05_scoring_path(case, monkeypatch):
     assert B.cobs_tcgen05_launches() == before          # and the default path does not
 
 
+# --- the exact-mass selector (OSA) -----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("case", ["cfg2_32k", "paged_g8_d64_ragged"])
+def test_exact_mass_selector_matches_oracle(case):
+    """cobs_exact_select against the oracle's direct summation (Eq. bg-defs) + group score + top-k."""
+    B = _binding()
+    if case == "cfg2_32k":
+        wl = WL["cfg2_32k"]
+    else:
+        lens = [32 * 21 + 7, 32 * 40, 19, 32 * 3]
+        wl = synth.Workload("osa", len(lens), 16, 2, 64, 32 * 40, 32, 16, rank=2, topk=5, window=70, summary_dtype="bf16",
+                            key_model="block_offset", planted=2, shuffle_pages=True, seed=51, seq_lens=lens)
+    inp = synth.generate(wl)
+    dev = to_dev(inp)
+    cfg = B.make_config(wl)
+    ws = B.alloc_workspace(cfg, "cuda")
+    nb, hkv, G, L = wl.batch, wl.n_kv_heads, wl.group, wl.block_size
+    sel = torch.full((nb, hkv, wl.topk), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((nb, hkv), -7, dtype=torch.int32, device="cuda")
+    scores = torch.zeros((nb, hkv, wl.max_blocks), dtype=torch.float32, device="cuda")
+    B.cobs_exact_select(cfg, dev["q"], B.make_kv(dev), sel, cnt, scores, ws)
+    assert B.cobs_read_status(ws) == 0
+    sel, cnt, scores = sel.cpu(), cnt.cpu(), scores.cpu().double().numpy()
+    for b in range(nb):
+        T = int(inp["seq_lens"][b])
+        n_sum = T // L
+        n_cand = O.window_start(T, wl.window, L) // L
+        for h in range(hkv):
+            K, _ = synth.unit_kv(inp, wl, b, h)
+            q = synth.unit_q(inp, wl, b, h).numpy()
+            assert int(cnt[b, h]) == min(wl.topk, n_cand)
+            if n_sum == 0:
+                continue
+            ref = O.group_scores(O.exact_log_masses(q, K.numpy(), L, n_sum))
+            err = np.max(np.abs(scores[b, h, :n_sum] - ref) / np.maximum(ref, 1e-30))
+            assert err <= SCORE_TOL, (b, h, err)
+            ok, msg, _ = check_selection(sel[b, h].tolist(), ref, n_cand, wl.topk)
+            assert ok, (b, h, msg)
+
+
 # --- shapes and edge cases ---------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("summary_dtype,scale_dtype", [("fp32", "fp32"), ("bf16", "fp32"), ("fp4", "fp32"),
