@@ -17,12 +17,12 @@ def _bf16_rows(gen, *shape):
     return torch.randn(*shape, generator=gen, dtype=torch.float32).to(torch.bfloat16)
 
 
-@pytest.mark.parametrize("summary_dtype", ["fp32", "fp4"])
-def test_decode_loop_matches_oracle_step_by_step(summary_dtype):
+@pytest.mark.parametrize("summary_dtype,P", [("fp32", 16), ("fp4", 16), ("bf16", 32)])
+def test_decode_loop_matches_oracle_step_by_step(summary_dtype, P):
     from paper_2607_09052_b200 import binding as B
     from paper_2607_09052_b200.decode_loop import DecodeLoop
 
-    L, P, D, G, Hkv = 32, 16, 64, 2, 2
+    L, D, G, Hkv = 32, 64, 2, 2
     start = [150, 97, 64]                        # mid-block, mid-block, exactly on a block boundary
     steps = 2 * L + 5
     wl = synth.Workload("loop", len(start), G * Hkv, Hkv, D, 12 * L, L, P, rank=4, topk=3, window=40,
