@@ -210,118 +210,131 @@ __device__ __forceinline__ bool wait_flag(const int *flag) {
 // ---------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void team_sync() { asm volatile("bar.sync 1, %0;\n" ::"n"(kSelThreads) : "memory"); }
 
-// Selection of one unit with everything in registers: thread t owns chunk t of the unit, i.e. blocks 16 t ...
-// 16 t + 15, whose (max, sum) pairs and t values it reads itself.  Needs n_chunks <= kFThreads and NB % 4 == 0.
-// Called by the 128 threads of the CTA's selection team (tid = index in the team).
+// Selection of one unit of at most 128 * BPT summarised blocks (BPT = 4, 8 or 16): thread t of the CTA's selection
+// team owns blocks BPT t ... BPT t + BPT - 1 (a part of chunk BPT t / 16, or all of chunk t), so that with few
+// blocks all four warps still hold keys and every loop over a thread's keys is short.  The global loads (the chunk
+// pairs, the maxima of this thread's own chunk parts, its t values of the first heads) are issued before the first
+// use: one round trip.  Needs NB % 4 == 0.
 // PPC: (max, sum) pairs per 16-block chunk and head left by the scoring path (1, or 4 = one per four blocks).
-template <int PPC>
-__device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, int tid) {
+template <int PPC, int BPT>
+__device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int tid) {
+  static_assert(BPT == 4 || BPT == 8 || BPT == 16, "blocks per thread");
+  static_assert(kSelWarps == 4, "one 16-byte read takes the four warps' words");
+  constexpr int NQ = BPT / 4;                    // groups of four blocks of a thread
+  constexpr int GB = (BPT == 16) ? 4 : 8;        // heads whose t values are in registers at a time
+  constexpr int CW = (BPT == 16) ? 2 : 1;        // words the three counts of a bisection round are packed in
   __shared__ float s_m[8][kSelWarps], s_s[8][kSelWarps];
-  __shared__ int s_cnt[2][3][kSelWarps];
-  __shared__ int s_scan[2][kSelWarps];
+  __shared__ __align__(16) int s_cnt[2][2][kSelWarps];
+  __shared__ int s_scan[kSelWarps];
   const int warp = tid >> 5, lane = tid & 31;
   const int G = p.G, NB = p.NB, cpu = (NB + 15) / 16, n_chunks = (n_sum + 15) / 16;
-  const bool mine = tid < n_chunks;
-  // ---- log-sum-exp per head from the chunk pairs -----------------------------------------------------------
+  const int b0 = tid * BPT, c_own = b0 >> 4, part0 = (b0 & 15) >> 2;
+  const bool mine = b0 < n_sum, loader = tid < n_chunks;
   const float2 *pp = reinterpret_cast<const float2 *>(p.lse_part) + (size_t)u * G * cpu * PPC;
-  float2 pr[8];
-  float msub[8][PPC];                            // PPC > 1: the maxima of the chunk's parts
+  const float *tu = p.e + (size_t)u * G * NB + b0;
+  // ---- loads -------------------------------------------------------------------------------------------------
+  float2 pr[8];                                  // (max, sum) of chunk `tid`, per head (threads below n_chunks)
+  float own_m[8][NQ];                            // max of the chunk part each of this thread's groups lies in
+  float4 x[GB][NQ];
+  auto load_t = [&](int g0) {
+#pragma unroll
+    for (int g = 0; g < GB; ++g)
+#pragma unroll
+      for (int q = 0; q < NQ; ++q)
+        x[g][q] = (g0 + g < G && b0 + 4 * q < n_sum) ? __ldcg(reinterpret_cast<const float4 *>(tu + (size_t)(g0 + g) * NB) + q)
+                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+  };
 #pragma unroll
   for (int g = 0; g < 8; ++g) {
     pr[g] = make_float2(-INFINITY, 0.f);
 #pragma unroll
-    for (int j = 0; j < PPC; ++j) msub[g][j] = -INFINITY;
-    if (g < G && mine) {
+    for (int q = 0; q < NQ; ++q) own_m[g][q] = -INFINITY;
+    if (g < G) {
       if (PPC == 1) {
-        pr[g] = __ldcg(pp + (size_t)g * cpu + tid);
+        if (loader) pr[g] = __ldcg(pp + (size_t)g * cpu + tid);
+        if (mine) {
+          const float m = (BPT == 16) ? pr[g].x : __ldcg(pp + (size_t)g * cpu + c_own).x;
+#pragma unroll
+          for (int q = 0; q < NQ; ++q) own_m[g][q] = m;
+        }
       } else {
         float2 part[PPC];
 #pragma unroll
-        for (int j = 0; j < PPC; j += 2) {
-          const float4 v = __ldcg(reinterpret_cast<const float4 *>(pp + ((size_t)g * cpu + tid) * PPC + j));
-          part[j] = make_float2(v.x, v.y);
-          part[j + (PPC > 1 ? 1 : 0)] = make_float2(v.z, v.w);
+        for (int j = 0; j < PPC; ++j) part[j] = make_float2(-INFINITY, 0.f);
+        if (loader) {
+#pragma unroll
+          for (int j = 0; j < PPC; j += 2) {
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(pp + ((size_t)g * cpu + tid) * PPC + j));
+            part[j] = make_float2(v.x, v.y);
+            part[j + (PPC > 1 ? 1 : 0)] = make_float2(v.z, v.w);
+          }
+          float m = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < PPC; ++j) m = fmaxf(m, part[j].x);
+          float sum = 0.f;
+#pragma unroll
+          for (int j = 0; j < PPC; ++j) sum += (part[j].x == -INFINITY) ? 0.f : part[j].y * __expf(part[j].x - m);
+          pr[g] = make_float2(m, sum);
         }
-        float m = -INFINITY;
+        if (mine) {
 #pragma unroll
-        for (int j = 0; j < PPC; ++j) { msub[g][j] = part[j].x; m = fmaxf(m, part[j].x); }
-        float sum = 0.f;
-#pragma unroll
-        for (int j = 0; j < PPC; ++j) sum += (part[j].x == -INFINITY) ? 0.f : part[j].y * __expf(part[j].x - m);
-        pr[g] = make_float2(m, sum);
+          for (int q = 0; q < NQ; ++q)
+            own_m[g][q] = (BPT == 16) ? part[q < PPC ? q : 0].x : __ldcg(pp + ((size_t)g * cpu + c_own) * PPC + part0 + q).x;
+        }
       }
     }
   }
+  load_t(0);
+  // ---- log-sum-exp per head: warp maximum by an integer reduction on the order-preserving bit pattern ----------
 #pragma unroll
   for (int g = 0; g < 8; ++g) {
     if (g < G) {
-      float m = pr[g].x, s = pr[g].y;
+      int im = __float_as_int(pr[g].x);
+      im ^= (im >> 31) & 0x7fffffff;
+      im = __reduce_max_sync(0xffffffffu, im);
+      im ^= (im >> 31) & 0x7fffffff;
+      const float M = __int_as_float(im);
+      float sum = (pr[g].x == -INFINITY) ? 0.f : pr[g].y * __expf(pr[g].x - M);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
-        const float nm = fmaxf(m, om);
-        s = (nm == -INFINITY) ? 0.f : s * __expf(m - nm) + os * __expf(om - nm);
-        m = nm;
-      }
-      if (lane == 0) { s_m[g][warp] = m; s_s[g][warp] = s; }
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) { s_m[g][warp] = M; s_s[g][warp] = sum; }
     }
   }
   COBS_SEL_STAMP(2);
   team_sync();
-  float w[8];                                    // exp(chunk max - lse) of this thread's chunk, per head
-  float wsub[8][PPC];                            // PPC > 1: exp(part max - lse)
+  // ---- scores of this thread's blocks: score_b = sum_g t[g][b] * exp(part max[g] - lse_g) -----------------------
+  float sc[BPT];
 #pragma unroll
-  for (int g = 0; g < 8; ++g) {
-    w[g] = 0.f;
+  for (int j = 0; j < BPT; ++j) sc[j] = 0.f;
 #pragma unroll
-    for (int j = 0; j < PPC; ++j) wsub[g][j] = 0.f;
-    if (g < G) {
-      float M = -INFINITY;
-#pragma unroll
-      for (int q = 0; q < kSelWarps; ++q) M = fmaxf(M, s_m[g][q]);
-      float S = 0.f;
-#pragma unroll
-      for (int q = 0; q < kSelWarps; ++q) S += (s_m[g][q] == -INFINITY) ? 0.f : s_s[g][q] * expf(s_m[g][q] - M);
-      const float lse = M + logf(S);
-      w[g] = mine ? expf(pr[g].x - lse) : 0.f;
-      if (PPC > 1) {
-#pragma unroll
-        for (int j = 0; j < PPC; ++j) wsub[g][j] = (mine && msub[g][j] != -INFINITY) ? expf(msub[g][j] - lse) : 0.f;
-      }
-    }
-  }
-  // ---- scores of this thread's 16 blocks ---------------------------------------------------------------------
-  float sc[16];
-#pragma unroll
-  for (int j = 0; j < 16; ++j) sc[j] = 0.f;
-  const float *tu = p.e + (size_t)u * G * NB + tid * 16;
-#pragma unroll
-  for (int g0 = 0; g0 < 8; g0 += 4) {
+  for (int g0 = 0; g0 < 8; g0 += GB) {
     if (g0 < G) {
-      float4 x[4][4];
+      if (g0 > 0) load_t(g0);
 #pragma unroll
-      for (int g = 0; g < 4; ++g)
+      for (int gg = 0; gg < GB; ++gg) {
+        const int g = g0 + gg;
+        if (g < G) {
+          float M = -INFINITY;
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-          x[g][q] = (g0 + g < G && mine && tid * 16 + 4 * q < n_sum)
-                        ? __ldcg(reinterpret_cast<const float4 *>(tu + (size_t)(g0 + g) * NB) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int q = 0; q < kSelWarps; ++q) M = fmaxf(M, s_m[g][q]);
+          float S = 0.f;
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        if (g0 + g < G) {
+          for (int q = 0; q < kSelWarps; ++q) S += (s_m[g][q] == -INFINITY) ? 0.f : s_s[g][q] * expf(s_m[g][q] - M);
+          const float lse = M + logf(S);
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float wg_ = (PPC == 4) ? wsub[g0 + g][PPC == 4 ? q : 0] : w[g0 + g];
-            sc[4 * q + 0] = fmaf(x[g][q].x, wg_, sc[4 * q + 0]); sc[4 * q + 1] = fmaf(x[g][q].y, wg_, sc[4 * q + 1]);
-            sc[4 * q + 2] = fmaf(x[g][q].z, wg_, sc[4 * q + 2]); sc[4 * q + 3] = fmaf(x[g][q].w, wg_, sc[4 * q + 3]);
+          for (int q = 0; q < NQ; ++q) {
+            const float wq = (own_m[g][q] != -INFINITY) ? expf(own_m[g][q] - lse) : 0.f;
+            sc[4 * q + 0] = fmaf(x[gg][q].x, wq, sc[4 * q + 0]); sc[4 * q + 1] = fmaf(x[gg][q].y, wq, sc[4 * q + 1]);
+            sc[4 * q + 2] = fmaf(x[gg][q].z, wq, sc[4 * q + 2]); sc[4 * q + 3] = fmaf(x[gg][q].w, wq, sc[4 * q + 3]);
           }
         }
       }
     }
   }
-  uint32_t keys[16];
+  uint32_t keys[BPT];
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    const int b = tid * 16 + j;
+  for (int j = 0; j < BPT; ++j) {
+    const int b = b0 + j;
     if (b >= n_sum) sc[j] = 0.f;                 // beyond the summarised blocks nothing was written
     if (p.scores && b < n_sum) p.scores[(size_t)u * NB + b] = sc[j];
     keys[j] = (b < n_cand) ? __float_as_uint(sc[j]) : 0u;
@@ -337,74 +350,76 @@ __device__ void select_unit_fast(const Params &p, int u, int n_sum, int n_cand, 
     return;
   }
   // k-th largest key by bisection on its bits (scores are >= 0, so their bit patterns order like integers):
-  // theta = the largest T with #(key >= T) >= k.  Bit 30 alone, then two bits per round (three trial values,
-  // one CTA barrier per round).
+  // theta = the largest T with #(key >= T) >= k.  Bit 30 alone, then two bits per round: three trial values, whose
+  // counts travel packed (11 bits each in one word while a team holds at most 1024 keys, else 16 bits each in two
+  // words): per round one or two warp reductions, one shared store per warp, one barrier, one 16-byte read per word.
+  constexpr int SH = (CW == 1) ? 11 : 16, SH2 = (CW == 1) ? 22 : 0;
   int par = 0;
-  auto cta_sums = [&](int c0, int c1, int c2, int &t0, int &t1, int &t2) {
-    c0 = __reduce_add_sync(0xffffffffu, c0); c1 = __reduce_add_sync(0xffffffffu, c1); c2 = __reduce_add_sync(0xffffffffu, c2);
-    if (lane == 0) { s_cnt[par][0][warp] = c0; s_cnt[par][1][warp] = c1; s_cnt[par][2][warp] = c2; }
+  auto cta_sum = [&](int c0, int c1, int &n0, int &n1) {
+    c0 = __reduce_add_sync(0xffffffffu, c0);
+    if (CW == 2) c1 = __reduce_add_sync(0xffffffffu, c1);
+    if (lane == 0) { s_cnt[par][0][warp] = c0; if (CW == 2) s_cnt[par][1][warp] = c1; }
     team_sync();
-    t0 = t1 = t2 = 0;
-#pragma unroll
-    for (int q = 0; q < kSelWarps; ++q) { t0 += s_cnt[par][0][q]; t1 += s_cnt[par][1][q]; t2 += s_cnt[par][2][q]; }
+    const int4 v = *reinterpret_cast<const int4 *>(&s_cnt[par][0][0]);
+    n0 = v.x + v.y + v.z + v.w;
+    n1 = 0;
+    if (CW == 2) {
+      const int4 w = *reinterpret_cast<const int4 *>(&s_cnt[par][1][0]);
+      n1 = w.x + w.y + w.z + w.w;
+    }
     par ^= 1;
   };
   uint32_t theta = 0u;
   {
     const uint32_t t = 1u << 30;
-    int c = 0, t0, t1, t2;
+    int c = 0, n0, n1;
 #pragma unroll
-    for (int j = 0; j < 16; ++j) c += (keys[j] >= t);
-    cta_sums(c, 0, 0, t0, t1, t2);
-    if (t0 >= k) theta = t;
+    for (int j = 0; j < BPT; ++j) c += (keys[j] >= t);
+    cta_sum(c, 0, n0, n1);
+    if (n0 >= k) theta = t;
   }
   for (int bit = 29; bit >= 1; bit -= 2) {
     const uint32_t ta = theta | (3u << (bit - 1)), tb = theta | (2u << (bit - 1)), tc = theta | (1u << (bit - 1));
-    int ca = 0, cb = 0, cc = 0, na, nb, nc;
+    int c0 = 0, c1 = 0, n0, n1;
 #pragma unroll
-    for (int j = 0; j < 16; ++j) { ca += (keys[j] >= ta); cb += (keys[j] >= tb); cc += (keys[j] >= tc); }
-    cta_sums(ca, cb, cc, na, nb, nc);
+    for (int j = 0; j < BPT; ++j) {
+      c0 += (keys[j] >= ta ? 1 : 0) + (keys[j] >= tb ? (1 << SH) : 0);
+      if (CW == 1) c0 += (keys[j] >= tc ? (1 << SH2) : 0);
+      else c1 += (keys[j] >= tc ? 1 : 0);
+    }
+    cta_sum(c0, c1, n0, n1);
+    const int na = n0 & ((1 << SH) - 1), nb = (n0 >> SH) & ((1 << SH) - 1), nc = (CW == 1) ? (n0 >> SH2) : n1;
     if (na >= k) theta = ta; else if (nb >= k) theta = tb; else if (nc >= k) theta = tc;
   }
   COBS_SEL_STAMP(4);
-  // keep every key above theta and the lowest-index `need_eq` keys equal to it, in index order
-  int n_gt_l = 0, n_eq = 0, d0, d1, d2;
+  // keep every key above theta and the lowest-index `need_eq` keys equal to it, in index order: one scan of the
+  // packed (above, equal) counts gives both the totals and this thread's position
+  int v = 0;
 #pragma unroll
-  for (int j = 0; j < 16; ++j) { n_gt_l += (keys[j] > theta); n_eq += (keys[j] == theta && tid * 16 + j < n_cand); }
-  cta_sums(n_gt_l, 0, 0, d0, d1, d2);
-  const int need_eq = k - d0;
-  auto cta_exclusive = [&](int v, int buf) -> int {
-    int inc = v;
+  for (int j = 0; j < BPT; ++j)
+    if (b0 + j < n_cand) v += (keys[j] > theta ? (1 << 16) : 0) + (keys[j] == theta ? 1 : 0);
+  int inc = v;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
-    }
-    if (lane == 31) s_scan[buf][warp] = inc;
-    team_sync();
-    int base = 0;
-#pragma unroll
-    for (int q = 0; q < kSelWarps; ++q) base += (q < warp) ? s_scan[buf][q] : 0;
-    return base + inc - v;
-  };
-  const int eq_base = cta_exclusive(n_eq, 0);
-  int eq_rank = eq_base, n_keep = 0;
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    if (tid * 16 + j < n_cand) {
-      if (keys[j] > theta) ++n_keep;
-      else if (keys[j] == theta) { if (eq_rank < need_eq) ++n_keep; ++eq_rank; }
-    }
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
   }
-  int pos = cta_exclusive(n_keep, 1);
-  eq_rank = eq_base;
+  if (lane == 31) s_scan[warp] = inc;
+  team_sync();
+  int base = 0, total = 0;
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    if (tid * 16 + j < n_cand) {
+  for (int q = 0; q < kSelWarps; ++q) { const int t = s_scan[q]; total += t; base += (q < warp) ? t : 0; }
+  const int need_eq = k - (total >> 16);
+  const int excl = base + inc - v;
+  int eq_rank = excl & 0xffff;
+  int pos = (excl >> 16) + min(eq_rank, need_eq);
+#pragma unroll
+  for (int j = 0; j < BPT; ++j) {
+    if (b0 + j < n_cand) {
       bool keep = false;
       if (keys[j] > theta) keep = true;
       else if (keys[j] == theta) { keep = eq_rank < need_eq; ++eq_rank; }
-      if (keep && pos < k) out[pos++] = tid * 16 + j;
+      if (keep && pos < k) out[pos++] = b0 + j;
     }
   }
   COBS_SEL_STAMP(5);
@@ -436,7 +451,9 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid, int c
     if (!ok) continue;                         // never scored: leave the unit unselected (its attention times out too)
     __threadfence();
     COBS_SEL_STAMP(0);
-    select_unit_fast<PPC>(p, u, n_sum, n_cand, tid);
+    if (n_sum <= kSelThreads * 4) select_unit<PPC, 4>(p, u, n_sum, n_cand, tid);
+    else if (n_sum <= kSelThreads * 8) select_unit<PPC, 8>(p, u, n_sum, n_cand, tid);
+    else select_unit<PPC, 16>(p, u, n_sum, n_cand, tid);
     __threadfence();
     team_sync();
     if (tid == 0) atomicExch(p.ctl_ready + u, 1);
