@@ -235,6 +235,61 @@ def test_ragged_lengths_and_degenerate_cases():
     run_stage_s(wl)
 
 
+def test_selection_exact_ties_for_every_blocks_per_thread_layout():
+    """The selection team spreads a unit's blocks 4, 8 or 16 per thread depending on the unit's block count.
+    Synthetic summaries with two kinds of block (every 16th block "hot", the rest "cold", identical within a kind)
+    make every score one of two values, exactly: the top-k must be all hot candidates plus the LOWEST-index cold
+    ones (ties -> lower index), for block counts on both sides of each layout boundary, in one batch."""
+    B = _binding()
+    L, D, G, NB, topk = 16, 64, 4, 2048, 48
+    n_sums = [3, 100, 511, 512, 513, 1024, 1025, 2047, 2048]
+    lens = [n * L + ((7 * i) % L if n < NB else 0) for i, n in enumerate(n_sums)]
+    wl = synth.Workload("ties", len(lens), G, 1, D, NB * L, L, 16, rank=2, topk=topk, window=70, summary_dtype="bf16",
+                        key_model="iid", seed=3, seq_lens=lens)
+    inp = synth.generate(wl)
+    gen = torch.Generator().manual_seed(5)
+    v = torch.randn(D, generator=gen)
+    q = (v[None, None, :] + 0.3 * torch.randn(len(lens), G, D, generator=gen)).to(torch.bfloat16)
+    inp["q"] = q
+    hot = (0.5 * v).to(torch.bfloat16)
+    cold = (-0.5 * v).to(torch.bfloat16)
+    f = (0.2 * torch.randn(2, D, generator=gen)).to(torch.bfloat16)
+    assert float((q.float() @ (hot.float() - cold.float())).min()) > 0        # hot beats cold for every head
+    dev = to_dev(inp)
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    mean_v, xi_v, _ = B.summary_views(cfg, summ)
+    is_hot = (torch.arange(NB) % 16 == 0)
+    mean_all = torch.where(is_hot[:, None], hot[None, :], cold[None, :])
+    mean_v[:, 0] = mean_all.cuda()[None]
+    xi_v[:, 0] = f.cuda()[None, None]
+    sel = torch.full((len(lens), 1, topk), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((len(lens), 1), -7, dtype=torch.int32, device="cuda")
+    B.cobs_score_select(cfg, dev["q"], summ, dev["seq_lens"], sel, cnt, None, ws)
+    out = torch.zeros((len(lens), G, D), dtype=torch.float32, device="cuda")
+    sel_f, cnt_f = torch.full_like(sel, -7), torch.full_like(cnt, -7)
+    B.cobs_decode_step(cfg, dev["q"], B.make_kv(dev), summ, out, None, sel_f, cnt_f, ws)
+    assert B.cobs_read_status(ws) == 0
+    sel, cnt, sel_f, cnt_f = sel.cpu(), cnt.cpu(), sel_f.cpu(), cnt_f.cpu()
+    mean_np, f_np = mean_all.double().numpy(), f.double().numpy()
+    for i, n_sum in enumerate(n_sums):
+        n_cand = O.window_start(lens[i], wl.window, L) // L
+        xi = np.broadcast_to(f_np[None], (n_sum, 2, D))
+        e = O.log_mass_estimates(q[i].double().numpy(), mean_np[:n_sum], xi, L)
+        score = O.group_scores(e)
+        assert len(set(score.tolist())) <= 2                                    # two values, exactly
+        ref = [int(x) for x in O.select_topk(score, n_cand, topk)]
+        k = min(topk, n_cand)
+        hot_c = [b for b in range(n_cand) if b % 16 == 0]
+        cold_c = [b for b in range(n_cand) if b % 16 != 0]
+        assert ref == sorted(hot_c[:k] + cold_c[:max(0, k - len(hot_c))])       # the oracle breaks ties by index
+        assert int(cnt[i, 0]) == k and int(cnt_f[i, 0]) == k
+        assert [int(x) for x in sel[i, 0, :k]] == ref, (n_sum, "cobs_score_select")
+        assert [int(x) for x in sel_f[i, 0, :k]] == ref, (n_sum, "cobs_decode_step")
+        assert all(int(x) == -1 for x in sel[i, 0, k:])
+
+
 def test_context_beyond_the_fused_selection_capacity():
     """4096 blocks per unit: more than the step kernel's selection team holds (2048), so scoring and selection
     take the generic kernels and only attention runs in the persistent kernel; same parity bar."""
