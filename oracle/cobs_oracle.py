@@ -27,6 +27,8 @@ in the paper's traffic and quantisation tables.  What the paper does not fix
 (tie order, window alignment, normaliser domain, eigenvector sign, the FP4
 scale formula and rounding rule) is a stated reading: parity unpinned by the
 paper for those choices; they are tested for self-consistency only.
+``adaptive_count`` / ``select_adaptive`` are an extension the paper does not
+define; they are pinned by a closed form and by brute force over subsets.
 """
 
 from __future__ import annotations
@@ -356,6 +358,38 @@ def select_topk(score, n_candidates, topk):
     cand = list(range(n_candidates))
     cand.sort(key=lambda b: (-score[b], b))
     return np.array(sorted(cand[:min(topk, n_candidates)]), dtype=np.int64)
+
+
+def adaptive_count(score, n_candidates, tau, k_min, k_max):
+    """Adaptive number of selected blocks.  NOT IN THE PAPER (the paper always keeps k blocks): an extension
+    built on the paper's dropped mass tau = sum of the normalised block masses outside the kept set S
+    (Background, the renormalisation paragraph before Eq. prop-gqa), applied to the group score of Eq. prop-gqa:
+
+      k_adapt = the smallest k such that the k largest candidate scores hold at least (1 - tau) of the
+                candidates' total score, clamped to [k_min, k_max] and to the number of candidates.
+
+    Ties in the ordering: lower index first, as in ``select_topk``.
+    """
+    s = np.asarray(score, dtype=np.float64)[:n_candidates]
+    if n_candidates == 0:
+        return 0
+    order = sorted(range(n_candidates), key=lambda b: (-s[b], b))
+    total = 0.0
+    for b in range(n_candidates):
+        total += s[b]
+    need = (1.0 - float(tau)) * total
+    k, cum = n_candidates, 0.0
+    for j, b in enumerate(order):
+        cum += s[b]
+        if cum >= need:
+            k = j + 1
+            break
+    return int(min(max(k, k_min), k_max, n_candidates))
+
+
+def select_adaptive(score, n_candidates, tau, k_min, k_max):
+    """The ``adaptive_count`` largest candidate scores, ascending index order (extension, not in the paper)."""
+    return select_topk(score, n_candidates, adaptive_count(score, n_candidates, tau, k_min, k_max))
 
 
 # ---------------------------------------------------------------------------

@@ -377,6 +377,45 @@ def test_selection_order_ties_and_window():
     assert list(toks) == list(range(0, 16)) + list(range(32, 48)) + list(range(112, 150))
 
 
+def test_adaptive_count_closed_form_and_brute_force():
+    """The adaptive block count (an extension, not in the paper).  (1) Geometric scores 2^-1, 2^-2, ... hold
+    1 - 2^-k of a total that tends to 1 in their k largest: k = ceil(log2(1 / tau)) up to the truncation of the
+    series.  (2) Brute force over all subsets of small random score vectors: the count is the size of the smallest
+    subset holding (1 - tau) of the total, and the selected set reaches that mass.  (3) Clamps and ties."""
+    import itertools
+    n = 40
+    score = np.array([2.0 ** -(j + 1) for j in range(n)])
+    rng = np.random.default_rng(3)
+    perm = rng.permutation(n)
+    shuffled = np.zeros(n)
+    shuffled[perm] = score                                   # the order in memory must not matter
+    for tau, want in ((0.5, 1), (0.3, 2), (0.25, 2), (0.2, 3), (0.01, 7), (1e-3, 10), (2.0 ** -20, 20)):
+        assert O.adaptive_count(shuffled, n, tau, 1, n) == want, tau
+        sel = O.select_adaptive(shuffled, n, tau, 1, n)
+        assert sorted(sel.tolist()) == sorted(perm[:want].tolist())
+    for trial in range(30):
+        m = int(rng.integers(3, 11))
+        s = rng.random(m) ** 3
+        tau = float(rng.choice([0.05, 0.2, 0.5]))
+        total = s.sum()
+        best = m
+        for size in range(1, m + 1):
+            if any(sum(s[list(c)]) >= (1 - tau) * total for c in itertools.combinations(range(m), size)):
+                best = size
+                break
+        k = O.adaptive_count(s, m, tau, 1, m)
+        assert k == best, (trial, k, best)
+        sel = O.select_adaptive(s, m, tau, 1, m)
+        assert s[sel].sum() >= (1 - tau) * total and len(sel) == k
+    s = np.array([5.0, 1.0, 1.0, 1.0, 1.0, 1.0])
+    assert O.adaptive_count(s, 6, 0.5, 1, 6) == 1                       # 5 of 10
+    assert O.adaptive_count(s, 6, 0.5, 3, 6) == 3                       # k_min
+    assert O.adaptive_count(s, 6, 0.0, 1, 4) == 4                       # k_max
+    assert O.adaptive_count(s, 4, 0.0, 1, 6) == 4                       # candidates only
+    assert O.select_adaptive(s, 6, 0.25, 1, 6).tolist() == [0, 1, 2, 3]  # 5 + 1 + 1 + 1 = 8 >= 7.5; ties -> low index
+    assert O.adaptive_count(s, 0, 0.1, 1, 6) == 0
+
+
 def test_fast_scores_equal_loop_scores_and_whole_step_brute_force():
     r = rng(15)
     G, D, L, NB, rnk, W, k = 2, 4, 4, 4, 2, 4, 2
