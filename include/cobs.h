@@ -193,6 +193,27 @@ int32_t cobs_exact_select(const cobs_config *cfg, const void *q, const cobs_kv *
                           float *scores_or_null, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Adaptive number of selected blocks: an EXTENSION, not in the paper (which always keeps topk blocks).  It applies
+ * the paper's dropped mass tau (the normalised block mass outside the kept set; Background, before Eq. prop-gqa) to
+ * the group score of Eq. prop-gqa: per (sequence, KV head),
+ *   k_adapt = the smallest k such that the k largest candidate scores hold at least (1 - tau) of the candidates'
+ *             total score, clamped to [k_min, topk] and to the number of candidates.
+ * Trims, in place, a selection made by cobs_score_select (or cobs_exact_select) with the same cfg:
+ *   scores    device, fp32 [batch][n_kv_heads][max_blocks]: the scores that call wrote (read only);
+ *   seq_lens  device, int32 [batch];
+ *   tau       in [0, 1); k_min >= 0;
+ *   sel_idx   device, int32 [batch][n_kv_heads][topk]: in, the topk best candidates in ascending index order;
+ *             out, the k_adapt best of them in ascending index order, the rest -1 (ties: lower index first);
+ *   sel_cnt   device, int32 [batch][n_kv_heads]: in, the entries in use; out, k_adapt.
+ * The result feeds cobs_sparse_decode, which reads sel_cnt entries per unit.  Sums are taken in double precision
+ * in a fixed order.  topk > 128: COBS_ERR_UNSUPPORTED.  An index outside the candidates is skipped and leaves
+ * COBS_ERR_BOUNDS in the status word.  The caller owns every buffer; the call is asynchronous on `stream`.
+ */
+int32_t cobs_adaptive_trim(const cobs_config *cfg, const float *scores, const int32_t *seq_lens, float tau,
+                           int32_t k_min, int32_t *sel_idx, int32_t *sel_cnt, void *workspace, size_t workspace_bytes,
+                           void *stream);
+
+/*
  * (d) Attention over the selected blocks and the window, one softmax over their union
  * (Eq. oracle-true restricted to the kept blocks and the window).
  * out [B][Hq][D] fp32; lse_or_null [B][Hq] fp32 = log of the softmax denominator (natural log).

@@ -24,6 +24,7 @@ EXPORTS = [
     "cobs_status_string", "cobs_padded_sub_dim", "cobs_summary_bytes", "cobs_workspace_bytes", "cobs_reset_status",
     "cobs_read_status", "cobs_build_summaries", "cobs_quantise_xi", "cobs_score_select", "cobs_sparse_decode",
     "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_tcgen05_launches", "cobs_sparse_decode_static", "cobs_append_token", "cobs_exact_select",
+    "cobs_adaptive_trim",
 ]
 
 
@@ -198,6 +199,15 @@ def cobs_exact_select(cfg: Config, q: torch.Tensor, kv: KV, sel_idx: torch.Tenso
     """Selection by exact block masses (reads every key): the quality reference for cobs_score_select."""
     _check(lib().cobs_exact_select(C.byref(cfg), _ptr(q), C.byref(kv), _ptr(sel_idx), _ptr(sel_cnt), _ptr(scores),
                                    _ptr(ws), C.c_size_t(ws.numel()), _stream(stream)), "cobs_exact_select")
+
+
+def cobs_adaptive_trim(cfg: Config, scores: torch.Tensor, seq_lens: torch.Tensor, tau: float, k_min: int,
+                       sel_idx: torch.Tensor, sel_cnt: torch.Tensor, ws: torch.Tensor, stream=None):
+    """Trim a selection, in place, to the smallest count that holds (1 - tau) of the candidates' total score
+    (an extension, not in the paper; see include/cobs.h)."""
+    _check(lib().cobs_adaptive_trim(C.byref(cfg), _ptr(scores), _ptr(seq_lens), C.c_float(tau), C.c_int32(k_min),
+                                    _ptr(sel_idx), _ptr(sel_cnt), _ptr(ws), C.c_size_t(ws.numel()), _stream(stream)),
+           "cobs_adaptive_trim")
 
 
 def cobs_sparse_decode(cfg: Config, q: torch.Tensor, kv: KV, sel_idx: torch.Tensor, sel_cnt: torch.Tensor,

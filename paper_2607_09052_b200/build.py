@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcobs.so")
-SOURCES = ["api.cu", "score_select.cu", "fused_step.cu", "summaries.cu", "exact_mass.cu"]
+SOURCES = ["api.cu", "score_select.cu", "fused_step.cu", "summaries.cu", "exact_mass.cu", "adaptive.cu"]
 
 
 def nvcc_path() -> str:

@@ -15,6 +15,7 @@ void count_tcgen05_launch() { g_tc_launches.fetch_add(1, std::memory_order_relax
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_select(const Params &p, cudaStream_t stream);
 cudaError_t launch_exact_mass(const Params &p, cudaStream_t stream);
+cudaError_t launch_adaptive_trim(const Params &p, float tau, int k_min, cudaStream_t stream);
 cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream);
 bool fused_score_supported(const Params &p);
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
@@ -342,6 +343,22 @@ int32_t cobs_exact_select(const cobs_config *cfg, const void *q, const cobs_kv *
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (launch_exact_mass(p, s) != cudaSuccess) return COBS_ERR_CUDA;
   return cuda_status(launch_select(p, s));
+}
+
+int32_t cobs_adaptive_trim(const cobs_config *cfg, const float *scores, const int32_t *seq_lens, float tau, int32_t k_min,
+                           int32_t *sel_idx, int32_t *sel_cnt, void *workspace, size_t workspace_bytes, void *stream) {
+  int32_t st = validate_config(cfg);
+  if (st != COBS_OK) return st;
+  if ((st = check_workspace(cfg, workspace, workspace_bytes)) != COBS_OK) return st;
+  if (!scores || !seq_lens || !sel_idx || !sel_cnt) return COBS_ERR_INVALID_ARG;
+  if (!(tau >= 0.f && tau < 1.f) || k_min < 0) return COBS_ERR_INVALID_ARG;
+  if (cfg->topk > 128) return COBS_ERR_UNSUPPORTED;
+  Params p;
+  fill_params(p, cfg, workspace);
+  p.seq_lens = seq_lens;
+  p.scores = const_cast<float *>(scores);
+  p.sel_idx = sel_idx; p.sel_cnt = sel_cnt;
+  return cuda_status(launch_adaptive_trim(p, tau, k_min, static_cast<cudaStream_t>(stream)));
 }
 
 int32_t cobs_sparse_decode(const cobs_config *cfg, const void *q, const cobs_kv *kv, const int32_t *sel_idx,

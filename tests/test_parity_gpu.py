@@ -290,6 +290,68 @@ def test_selection_exact_ties_for_every_blocks_per_thread_layout():
         assert all(int(x) == -1 for x in sel[i, 0, k:])
 
 
+@pytest.mark.parametrize("key_model,planted", [("block_offset", 4), ("iid", 0)])
+def test_adaptive_block_count_extension(key_model, planted):
+    """cobs_score_select -> cobs_adaptive_trim -> cobs_sparse_decode against the oracle's adaptive_count /
+    select_adaptive (an extension, not in the paper).  The count may differ from the oracle's only where the kept
+    mass is within 5e-5 of the threshold (fp32 scores on the device, fp64 in the oracle): it must lie between the
+    oracle's counts for tau +- 5e-5; the kept set is then checked with the usual tie band, and the attention output
+    on the device's own trimmed selection against the oracle's attention over the same blocks."""
+    B = _binding()
+    L, topk, k_min = 64, 64, 3
+    lens = [L * 96, L * 50 + 9, L * 3, L * 20 + 63]
+    wl = synth.Workload("adapt", len(lens), 8, 2, 128, L * 96, L, 16, rank=4, topk=topk, window=130,
+                        summary_dtype="bf16", key_model=key_model, planted=planted, shuffle_pages=True, seed=21,
+                        seq_lens=lens)
+    inp = synth.generate(wl)
+    dev = to_dev(inp)
+    cfg = B.make_config(wl)
+    kv = B.make_kv(dev)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    nb, hq, hkv, G, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.group, wl.head_dim
+    ref = {}
+    for b in range(nb):
+        for h in range(hkv):
+            st = oracle_unit_summaries(wl, inp, b, h)
+            upload_unit_summaries(B, cfg, summ, b, h, st)
+            ref[(b, h)] = oracle_unit_step(wl, inp, b, h, st)
+    scores = torch.zeros((nb, hkv, wl.max_blocks), dtype=torch.float32, device="cuda")
+    counts = []
+    for tau in (0.5, 0.1, 0.01, 0.0):
+        tau32 = float(np.float32(tau))
+        sel = torch.full((nb, hkv, topk), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((nb, hkv), -7, dtype=torch.int32, device="cuda")
+        B.cobs_score_select(cfg, dev["q"], summ, dev["seq_lens"], sel, cnt, scores, ws)
+        B.cobs_adaptive_trim(cfg, scores, dev["seq_lens"], tau32, k_min, sel, cnt, ws)
+        out = torch.zeros((nb, hq, D), dtype=torch.float32, device="cuda")
+        lse = torch.zeros((nb, hq), dtype=torch.float32, device="cuda")
+        B.cobs_sparse_decode(cfg, dev["q"], kv, sel, cnt, out, lse, ws)
+        assert B.cobs_read_status(ws) == 0
+        sel_c, cnt_c, out_c, lse_c = sel.cpu(), cnt.cpu(), out.cpu().numpy(), lse.cpu().numpy()
+        for (b, h), r in ref.items():
+            n_cand = O.window_start(lens[b], wl.window, L) // L
+            k_gpu = int(cnt_c[b, h])
+            k_lo = O.adaptive_count(r["score"], n_cand, min(tau32 + 5e-5, 1.0), k_min, topk)
+            k_hi = O.adaptive_count(r["score"], n_cand, max(tau32 - 5e-5, 0.0), k_min, topk)
+            assert k_lo <= k_gpu <= k_hi, (tau, b, h, k_gpu, k_lo, k_hi)
+            gpu_sel = [int(x) for x in sel_c[b, h, :k_gpu]]
+            assert all(int(x) == -1 for x in sel_c[b, h, k_gpu:])
+            ok, msg, _ = check_selection(gpu_sel, r["score"], n_cand, k_gpu)
+            assert ok, (tau, b, h, msg)
+            ref_out, ref_lse = oracle_attend(wl, inp, b, h, gpu_sel)
+            hs = slice(h * G, (h + 1) * G)
+            assert np.all(out_rel_err(out_c[b, hs], ref_out) <= OUT_TOL), (tau, b, h)
+            assert np.allclose(lse_c[b, hs], ref_lse, atol=2e-3, rtol=0)
+            counts.append((tau, k_gpu, n_cand))
+    # the rule does something: tau = 0 keeps everything it may, a large tau keeps fewer blocks where there are many
+    assert all(k == min(topk, n) for t, k, n in counts if t == 0.0)
+    assert any(k < min(topk, n) for t, k, n in counts if t == 0.5 and n > topk)
+    if planted:
+        # four planted blocks hold most of the mass: half of it needs only a few blocks
+        assert all(k <= 8 for t, k, n in counts if t == 0.5 and n > topk)
+
+
 def test_context_beyond_the_fused_selection_capacity():
     """4096 blocks per unit: more than the step kernel's selection team holds (2048), so scoring and selection
     take the generic kernels and only attention runs in the persistent kernel; same parity bar."""
