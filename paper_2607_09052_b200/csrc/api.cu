@@ -420,9 +420,22 @@ int32_t cobs_decode_step_host(const cobs_config *cfg, const void *q_host, const 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t n = (size_t)cfg->batch * cfg->n_q_heads * cfg->head_dim;
   if (cudaMemcpyAsync(q_dev, q_host, n * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return COBS_ERR_CUDA;
-  st = cobs_decode_step(cfg, q_dev, kv, summ, out_dev, nullptr, nullptr, nullptr, workspace, workspace_bytes, stream);
+  // Pinned, device-mapped output memory: the merge writes its rows straight into it (posted writes over PCIe, 256 KB
+  // spread over the tail of the kernel), which saves a device-to-host copy and its latency after the kernel.  Any
+  // other host memory goes through the staging buffer.
+  float *out_direct = nullptr;
+  {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, out_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+        attr.devicePointer != nullptr && aligned16(attr.devicePointer))
+      out_direct = static_cast<float *>(attr.devicePointer);
+    else
+      (void)cudaGetLastError();                  // unregistered host memory reports an error on some drivers: clear it
+  }
+  st = cobs_decode_step(cfg, q_dev, kv, summ, out_direct ? out_direct : out_dev, nullptr, nullptr, nullptr, workspace,
+                        workspace_bytes, stream);
   if (st != COBS_OK) return st;
-  if (cudaMemcpyAsync(out_host, out_dev, n * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+  if (!out_direct && cudaMemcpyAsync(out_host, out_dev, n * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
     return COBS_ERR_CUDA;
   if (sel_idx_host_or_null) {
     const size_t units = (size_t)cfg->batch * cfg->n_kv_heads;

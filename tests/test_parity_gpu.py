@@ -412,6 +412,12 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     cnt_h = torch.zeros((1, 8), dtype=torch.int32).pin_memory()
     B.cobs_decode_step_host(cfg, q_h, kv, summ, out_h, sel_h, cnt_h, ws)
     assert torch.equal(out_h, out_d.cpu()) and torch.equal(sel_h, sel_d.cpu()) and torch.equal(cnt_h, cnt_d.cpu())
+    # pinned output memory is written by the kernel itself; pageable memory goes through the staging buffer
+    out_p = torch.zeros((1, 32, 128), dtype=torch.float32)
+    assert not out_p.is_pinned()
+    B.cobs_decode_step_host(cfg, q_h, kv, summ, out_p, None, None, ws)
+    assert torch.equal(out_p, out_d.cpu())
+    assert B.cobs_read_status(ws) == 0
 
 
 # --- quantiser (bit exact) -----------------------------------------------------------------------------------
