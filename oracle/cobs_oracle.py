@@ -27,7 +27,9 @@ in the paper's traffic and quantisation tables.  What the paper does not fix
 (tie order, window alignment, normaliser domain, eigenvector sign, the FP4
 scale formula and rounding rule) is a stated reading: parity unpinned by the
 paper for those choices; they are tested for self-consistency only.
-``adaptive_count`` / ``select_adaptive`` are an extension the paper does not
+``block_skew`` / ``log_mass_estimates_skew`` (the paper's diagonal-skew variant) are
+pinned by the third derivative of the exact log mass and by the order of the
+remaining error.  ``adaptive_count`` / ``select_adaptive`` are an extension the paper does not
 define; they are pinned by a closed form and by brute force over subsets.
 """
 
@@ -217,6 +219,58 @@ def build_summaries(K, block_size, rank, u_q=None, n_blocks=None):
     for b in range(nb):
         mean[b], xi[b], lam[b] = scaled_eigenvectors_gram(K[b * L:(b + 1) * L], rank, u_q)
     return mean, xi, lam
+
+
+def block_skew(k_block, xi):
+    """Diagonal of the third cumulant in the stored eigenbasis (Appendix, "Cheap diagonal skew").
+
+    For every stored factor xi_i = sqrt(lam_i) u_i of a block (full-space descriptor):
+      g_i = 1/L * sum_{t in b} (u_i . (k_t - kbar))^3 .
+    The correction to the block log-score is 1/6 * sum_i (u_i . q')^3 g_i.  With u_i . q' = (xi_i . q') / sqrt(lam_i)
+    it equals 1/6 * sum_i c_i (xi_i . q')^3 for c_i = g_i / lam_i^(3/2), which is the scalar returned (and stored)
+    per factor; a null factor (lam_i = 0) gets 0.
+    k_block [L, D], xi [r, D] -> c [r].
+    """
+    k_block = np.asarray(k_block, dtype=np.float64)
+    xi = np.asarray(xi, dtype=np.float64)
+    L = k_block.shape[0]
+    kbar = k_block.sum(axis=0) / L
+    c = np.zeros(xi.shape[0])
+    for i in range(xi.shape[0]):
+        lam = float(xi[i] @ xi[i])
+        if lam == 0.0:
+            continue
+        u = xi[i] / np.sqrt(lam)
+        g = 0.0
+        for t in range(L):
+            g += float(u @ (k_block[t] - kbar)) ** 3
+        g /= L
+        c[i] = g / lam ** 1.5
+    return c
+
+
+def build_skew(K, block_size, xi):
+    """``block_skew`` for every summarised block: K [T, D], xi [NB, r, D] (exact factors) -> [NB, r]."""
+    K = np.asarray(K, dtype=np.float64)
+    L = block_size
+    return np.stack([block_skew(K[b * L:(b + 1) * L], xi[b]) for b in range(xi.shape[0])]) if xi.shape[0] else np.zeros((0, xi.shape[1]))
+
+
+def log_mass_estimates_skew(q, mean, xi, skew, block_size):
+    """Second-order estimate plus the diagonal third-cumulant term (Appendix, "Cheap diagonal skew"):
+      e[g, b] = ln L + q'_g . kbar_b + 1/2 sum_i (xi_{b,i} . q'_g)^2 + 1/6 sum_i c_{b,i} (xi_{b,i} . q'_g)^3 .
+    mean [NB, D], xi [NB, r, D] as stored, skew [NB, r] as stored (binary32 values)."""
+    qs = scale_query(q)
+    G, nb = qs.shape[0], mean.shape[0]
+    e = np.zeros((G, nb))
+    for g in range(G):
+        for b in range(nb):
+            val = np.log(block_size) + qs[g] @ mean[b]
+            for i in range(xi.shape[1]):
+                d = xi[b, i] @ qs[g]
+                val += 0.5 * d * d + skew[b, i] * d * d * d / 6.0
+            e[g, b] = val
+    return e
 
 
 def store_summaries(mean, xi, summary_dtype, scale_dtype="fp32"):

@@ -377,6 +377,55 @@ def test_selection_order_ties_and_window():
     assert list(toks) == list(range(0, 16)) + list(range(32, 48)) + list(range(112, 150))
 
 
+def test_skew_is_third_derivative_of_exact_log_mass_and_cuts_the_error_order():
+    """Diagonal skew (Appendix, "Cheap diagonal skew").  (1) g_i is the third cumulant of the keys projected on
+    u_i, i.e. the third derivative at 0 of t -> ln m_b(t u_i): checked by a central finite difference of the EXACT
+    log mass.  (2) For a block whose keys vary along one direction only the diagonal is the whole third-order
+    tensor: the estimate with the skew term is exact to O(t^4) where the second-order one is exact to O(t^3)
+    (halving t divides the errors by ~16 and ~8 respectively), and the second-order error / t^3 tends to g / 6."""
+    rng = np.random.default_rng(11)
+    L, D, r = 32, 16, 3
+    K = rng.standard_normal((L, D)) * np.array([2.0, 1.5, 1.2] + [0.3] * (D - 3))
+    K[:, 0] = np.abs(K[:, 0]) ** 1.5                        # a skewed coordinate
+    mean, xi, lam = O.scaled_eigenvectors_gram(K, r)
+    c = O.block_skew(K, xi)
+    for i in range(r):
+        u = xi[i] / np.sqrt(lam[i])
+        f = lambda t: O.exact_log_masses((t * u * np.sqrt(D))[None, :], K, L, 1)[0, 0]
+        h = 0.02
+        third = (f(2 * h) - 2 * f(h) + 2 * f(-h) - f(-2 * h)) / (2 * h ** 3)
+        g = c[i] * lam[i] ** 1.5
+        assert abs(third - g) <= 2e-3 * max(1.0, abs(g)), (i, third, g)
+    assert abs(c[0]) > 1e-3                                  # the skewed direction has a skew to speak of
+    # rank-one block: k_t = kbar + a_t v
+    v = rng.standard_normal(D)
+    v /= np.linalg.norm(v)
+    a = rng.gamma(2.0, 1.0, L)
+    K1 = 0.3 * rng.standard_normal(D)[None, :] + a[:, None] * v[None, :]
+    mean1, xi1, lam1 = O.scaled_eigenvectors_gram(K1, 1)
+    c1 = O.block_skew(K1, xi1)
+    g1 = c1[0] * lam1[0] ** 1.5
+    sign = np.sign(xi1[0] @ v)
+    errs2, errs3 = [], []
+    for t in (0.2, 0.1, 0.05):
+        q = (t * sign * v * np.sqrt(D))[None, :]
+        exact = O.exact_log_masses(q, K1, L, 1)[0, 0]
+        e2 = O.log_mass_estimates(q, mean1[None], xi1[None], L)[0, 0]
+        e3 = O.log_mass_estimates_skew(q, mean1[None], xi1[None], c1[None], L)[0, 0]
+        errs2.append(exact - e2)
+        errs3.append(exact - e3)
+    assert 6.5 < errs2[0] / errs2[1] < 9.5 and 6.5 < errs2[1] / errs2[2] < 9.5       # O(t^3)
+    assert 10.0 < errs3[0] / errs3[1] < 22.0 and 10.0 < errs3[1] / errs3[2] < 22.0   # O(t^4)
+    assert all(abs(e3) < 0.01 * abs(e2) for e2, e3 in zip(errs2, errs3))
+    assert abs(errs2[2] / 0.05 ** 3 - g1 / 6.0) <= 0.05 * abs(g1 / 6.0)
+    # a null factor stores 0; sign of the factor does not matter for the correction
+    assert O.block_skew(K1, np.zeros((1, D)))[0] == 0.0
+    qq = rng.standard_normal((2, D))
+    ea = O.log_mass_estimates_skew(qq, mean[None], xi[None], c[None], L)
+    eb = O.log_mass_estimates_skew(qq, mean[None], -xi[None], O.block_skew(K, -xi)[None], L)
+    assert np.allclose(ea, eb, rtol=0, atol=1e-12)
+
+
 def test_adaptive_count_closed_form_and_brute_force():
     """The adaptive block count (an extension, not in the paper).  (1) Geometric scores 2^-1, 2^-2, ... hold
     1 - 2^-k of a total that tends to 1 in their k largest: k = ceil(log2(1 / tau)) up to the truncation of the
