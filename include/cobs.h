@@ -108,7 +108,18 @@ typedef struct {
   void *xi;
   void *scale;
   const float *u_q;
+  float *skew;                /* NULL, or [B][Hkv][NB][r] fp32: the diagonal-skew variant (see below) */
 } cobs_summaries;
+
+/*
+ * Diagonal-skew variant (paper: Appendix, "Cheap diagonal skew"; it reports that the term hurts at r <= 8 and stops
+ * at the covariance, so this is off unless `skew` is given).  One scalar per stored factor xi_i = sqrt(lam_i) u_i,
+ *   c_i = g_i / lam_i^(3/2),   g_i = 1/L sum_{t in b} (u_i . (k_t - kbar))^3   (0 for a null factor),
+ * adds 1/6 sum_i c_i (xi_i . q')^3 (= 1/6 sum_i (u_i . q')^3 g_i) to the block's log-mass estimate.
+ * With skew != NULL: cobs_build_summaries writes the scalars (from the unrounded factors), cobs_score_select and
+ * cobs_decode_step add the term; scoring then runs in the generic kernels, not in the one-launch step.  Full-space
+ * descriptors only (sub_dim == 0), rank >= 1: otherwise COBS_ERR_UNSUPPORTED.
+ */
 
 const char *cobs_status_string(int32_t status);
 

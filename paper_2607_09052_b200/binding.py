@@ -46,7 +46,8 @@ class KV(C.Structure):
 
 
 class Summaries(C.Structure):
-    _fields_ = [("mean", C.c_void_p), ("xi", C.c_void_p), ("scale", C.c_void_p), ("u_q", C.c_void_p)]
+    _fields_ = [("mean", C.c_void_p), ("xi", C.c_void_p), ("scale", C.c_void_p), ("u_q", C.c_void_p),
+                ("skew", C.c_void_p)]
 
 
 _lib = None
@@ -130,17 +131,21 @@ def cobs_workspace_bytes(cfg: Config) -> int:
 class SummaryBuffers:
     """Device buffers for the summary arrays of one workload, sized by the library."""
 
-    def __init__(self, cfg: Config, device, u_q: Optional[torch.Tensor] = None):
+    def __init__(self, cfg: Config, device, u_q: Optional[torch.Tensor] = None, skew: bool = False):
         mb, xb, sb = cobs_summary_bytes(cfg)
         self.mean = torch.zeros(max(mb, 16), dtype=torch.uint8, device=device)
         self.xi = torch.zeros(max(xb, 16), dtype=torch.uint8, device=device)
         self.scale = torch.zeros(max(sb, 16), dtype=torch.uint8, device=device)
         self.u_q = u_q
+        # the diagonal-skew variant: one fp32 scalar per stored factor, [B][Hkv][NB][r]
+        self.skew = (torch.zeros((cfg.batch, cfg.n_kv_heads, cfg.max_blocks, max(cfg.rank, 1)), dtype=torch.float32,
+                                 device=device) if skew else None)
         self.nbytes = (mb, xb, sb)
 
     def struct(self) -> Summaries:
         return Summaries(self.mean.data_ptr(), self.xi.data_ptr(), self.scale.data_ptr(),
-                         self.u_q.data_ptr() if self.u_q is not None else 0)
+                         self.u_q.data_ptr() if self.u_q is not None else 0,
+                         self.skew.data_ptr() if self.skew is not None else 0)
 
 
 def alloc_workspace(cfg: Config, device) -> torch.Tensor:

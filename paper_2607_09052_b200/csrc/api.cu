@@ -162,6 +162,11 @@ static int32_t set_summaries(Params &p, const cobs_config *c, const cobs_summari
   if (c->sub_dim != 0 && (!s->u_q || !aligned16(s->u_q))) return COBS_ERR_INVALID_ARG;
   p.mean = s->mean; p.xi = s->xi; p.scale = s->scale;
   p.u_q = c->sub_dim ? s->u_q : nullptr;
+  if (s->skew) {
+    if (c->sub_dim != 0 || c->rank < 1) return COBS_ERR_UNSUPPORTED;
+    if (!aligned16(s->skew)) return COBS_ERR_INVALID_ARG;
+    p.skew = s->skew;
+  }
   return COBS_OK;
 }
 

@@ -30,6 +30,7 @@ struct Params {
   // summaries
   void *mean, *xi, *scale;
   const float *u_q;
+  float *skew;                // optional [B][Hkv][NB][r] fp32: third-cumulant scalar per stored factor (full-space descriptors)
   // workspace pieces
   int32_t *status;
   int *ctl_done;              // CTAs of the persistent kernel that have finished

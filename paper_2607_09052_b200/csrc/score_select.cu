@@ -1,6 +1,7 @@
 // Steps (b) and (c): second-order block scores from the stored summaries, GQA group score, top-k.
 //
 //   e[g][b]  = ln L + q'_g . mean_b + 1/2 sum_i (xi_{b,i} . q~_g)^2      (Eq. trunc with Eq. gram)
+//              [+ 1/6 sum_i c_{b,i} (xi_{b,i} . q'_g)^3 when skew scalars are given: Appendix, Cheap diagonal skew]
 //   score[b] = sum_g exp(e[g][b] - logsumexp_b' e[g][b'])                (Eq. gqa-secondorder)
 //   selection: k largest scores among the candidate blocks, lower index on ties, ascending output.
 #include "common.cuh"
@@ -92,10 +93,11 @@ __global__ void __launch_bounds__(256) score_generic_kernel(Params p, int blocks
 #pragma unroll
         for (int g = 0; g < G; ++g) acc[g] = fmaf(x, qt[g * p.Ds_pad + j], acc[g]);
       }
+      const float c6 = p.skew ? p.skew[rec * p.r + i] * (1.0f / 3.0f) : 0.f;   // (c / 6) / (1 / 2): folded into `second`
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         float d = warp_sum(acc[g]) * sc;
-        second[g] = fmaf(d, d, second[g]);
+        second[g] = fmaf(d * d, fmaf(c6, d, 1.0f), second[g]);                 // d^2 + (c / 3) d^3
       }
     }
     if (lane < G) {

@@ -311,6 +311,48 @@ __global__ void __launch_bounds__(kBuildThreads) build_kernel(Params p, int bloc
                         p.scale, v, p.scale_dtype, lane);
     }
   }
+
+  // ---- diagonal of the third cumulant in the stored eigenbasis (Appendix, Cheap diagonal skew) -------------------
+  // c_i = g_i / lam_i^(3/2) with g_i = 1/L sum_t (u_i . (k_t - kbar))^3 and xi_i = sqrt(lam_i) u_i, i.e.
+  // c_i = [1/L sum_t p_t^3] / lam_i^3 for p_t = xi_i . (k_t - kbar).  The projections are taken on the raw keys and
+  // centred afterwards (xi_i . kbar is their mean), from the unrounded, sign-fixed factors.  Full space only (Dk = D).
+  if (p.skew) {
+    __syncthreads();
+    float *proj = Kc;                            // [r][L]: the rotated rows are no longer needed
+    for (int t = warp; t < L; t += NW) {
+      const int tok = blk * L + t;
+      const int pg = p.page_table[(size_t)b_idx * p.mpp + tok / p.P];
+      const bool okp = pg >= 0 && pg < p.n_pages;           // a bad page was reported when the keys were loaded
+      const __nv_bfloat16 *kr = p.k_pages + (((size_t)(okp ? pg : 0) * p.Hkv + h) * p.P + (tok % p.P)) * D;
+      float kreg[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) kreg[i] = (okp && lane + 32 * i < D) ? __bfloat162float(kr[lane + 32 * i]) : 0.f;
+      for (int f = 0; f < p.r; ++f) {
+        float a = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (lane + 32 * i < D) a = fmaf(kreg[i], xi_s[f * Dk + lane + 32 * i], a);
+        a = warp_sum(a);
+        if (lane == 0) proj[f * L + t] = a;
+      }
+    }
+    __syncthreads();
+    for (int f = warp; f < p.r; f += NW) {
+      const float *row = xi_s + f * Dk;
+      float lam = 0.f, sum = 0.f;
+      for (int j = lane; j < Dk; j += 32) lam = fmaf(row[j], row[j], lam);
+      for (int t = lane; t < L; t += 32) sum += proj[f * L + t];
+      lam = warp_sum(lam);
+      const float m = warp_sum(sum) / (float)L;
+      float c3 = 0.f;
+      for (int t = lane; t < L; t += 32) {
+        const float x = proj[f * L + t] - m;
+        c3 = fmaf(x * x, x, c3);
+      }
+      c3 = warp_sum(c3) / (float)L;
+      if (lane == 0) p.skew[rec * p.r + f] = (top[f] >= 0 && lam > 0.f) ? c3 / (lam * lam * lam) : 0.f;
+    }
+  }
 }
 
 size_t build_smem_bytes(const Params &p) {

@@ -352,6 +352,103 @@ def test_adaptive_block_count_extension(key_model, planted):
         assert all(k <= 8 for t, k, n in counts if t == 0.5 and n > topk)
 
 
+@pytest.mark.parametrize("summary_dtype", ["bf16", "fp4"])
+def test_diagonal_skew_variant_scores_and_step(summary_dtype):
+    """The paper's diagonal-skew variant (Appendix, Cheap diagonal skew): with skew scalars given, scores carry the
+    cubic term.  Oracle summaries and oracle skew scalars are uploaded bit for bit; scores, selection and the step's
+    output are compared with the oracle's skew estimate."""
+    B = _binding()
+    L = 32
+    lens = [L * 40, L * 23 + 5, L * 2]
+    wl = synth.Workload("skew", len(lens), 8, 2, 64, L * 40, L, 16, rank=4, topk=6, window=70,
+                        summary_dtype=summary_dtype, key_model="block_offset", planted=2, shuffle_pages=True, seed=9,
+                        seq_lens=lens)
+    inp = synth.generate(wl)
+    dev = to_dev(inp)
+    cfg = B.make_config(wl)
+    kv = B.make_kv(dev)
+    summ = B.SummaryBuffers(cfg, "cuda", skew=True)
+    ws = B.alloc_workspace(cfg, "cuda")
+    nb, hq, hkv, G, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.group, wl.head_dim
+    ref, differs = {}, 0
+    for b in range(nb):
+        for h in range(hkv):
+            st = oracle_unit_summaries(wl, inp, b, h)
+            upload_unit_summaries(B, cfg, summ, b, h, st)
+            K, _ = synth.unit_kv(inp, wl, b, h)
+            n = st["mean"].shape[0]
+            c = O.build_skew(K.numpy(), L, st["xi_exact"]).astype(np.float32)
+            if n:
+                summ.skew[b, h, :n] = torch.from_numpy(c).cuda()
+            q = synth.unit_q(inp, wl, b, h).numpy()
+            e = O.log_mass_estimates_skew(q, st["mean"], st["xi"], c.astype(np.float64), L)
+            score = O.group_scores(e) if n else np.zeros(0)
+            plain = O.group_scores(O.log_mass_estimates(q, st["mean"], st["xi"], L)) if n else np.zeros(0)
+            differs += int(np.sum(np.abs(score - plain) > 1e-3 * np.maximum(plain, 1e-30)))
+            ref[(b, h)] = score
+    assert differs > 0                                            # the cubic term moves the scores
+    sel = torch.full((nb, hkv, wl.topk), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((nb, hkv), -7, dtype=torch.int32, device="cuda")
+    scores = torch.zeros((nb, hkv, wl.max_blocks), dtype=torch.float32, device="cuda")
+    B.cobs_score_select(cfg, dev["q"], summ, dev["seq_lens"], sel, cnt, scores, ws)
+    out = torch.zeros((nb, hq, D), dtype=torch.float32, device="cuda")
+    lse = torch.zeros((nb, hq), dtype=torch.float32, device="cuda")
+    sel_f, cnt_f = torch.full_like(sel, -7), torch.full_like(cnt, -7)
+    B.cobs_decode_step(cfg, dev["q"], kv, summ, out, lse, sel_f, cnt_f, ws)
+    assert B.cobs_read_status(ws) == 0
+    sel, cnt, scores = sel.cpu(), cnt.cpu(), scores.cpu().double().numpy()
+    out, lse, sel_f, cnt_f = out.cpu().numpy(), lse.cpu().numpy(), sel_f.cpu(), cnt_f.cpu()
+    for (b, h), score in ref.items():
+        n_sum = lens[b] // L
+        n_cand = O.window_start(lens[b], wl.window, L) // L
+        if n_sum:
+            err = np.max(np.abs(scores[b, h, :n_sum] - score) / np.maximum(score, 1e-30))
+            assert err <= SCORE_TOL, (b, h, err)
+        ok, msg, _ = check_selection(sel[b, h].tolist(), score, n_cand, wl.topk)
+        assert ok, (b, h, msg)
+        assert torch.equal(sel_f[b, h], sel[b, h]) and int(cnt_f[b, h]) == int(cnt[b, h]) == min(wl.topk, n_cand)
+        ref_out, ref_lse = oracle_attend(wl, inp, b, h, [int(x) for x in sel_f[b, h] if x >= 0])
+        hs = slice(h * G, (h + 1) * G)
+        assert np.all(out_rel_err(out[b, hs], ref_out) <= OUT_TOL), (b, h)
+        assert np.allclose(lse[b, hs], ref_lse, atol=2e-3, rtol=0)
+
+
+def test_builder_writes_skew_scalars():
+    """cobs_build_summaries with a skew buffer (fp32 summaries): the scalars against the oracle's block_skew, directly
+    where the factor's eigenvalue is well separated (elsewhere the eigenvector itself is not unique to rounding), and
+    for every factor against block_skew evaluated on the factor the device stored."""
+    B = _binding()
+    L, D, r = 32, 64, 4
+    wl = synth.Workload("skewb", 2, 4, 2, D, L * 12, L, 16, rank=r, topk=2, window=40, summary_dtype="fp32",
+                        key_model="lowrank16", shuffle_pages=True, seed=17, seq_lens=[L * 12, L * 7 + 3])
+    inp = synth.generate(wl)
+    dev = to_dev(inp)
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda", skew=True)
+    ws = B.alloc_workspace(cfg, "cuda")
+    B.cobs_build_summaries(cfg, B.make_kv(dev), 0, wl.max_blocks, summ, ws)
+    assert B.cobs_read_status(ws) == 0
+    _, xi_v, _ = B.summary_views(cfg, summ)
+    xi_gpu, skew_gpu = xi_v.cpu().double().numpy(), summ.skew.cpu().double().numpy()
+    direct = 0
+    for b in range(wl.batch):
+        for h in range(wl.n_kv_heads):
+            K, _ = synth.unit_kv(inp, wl, b, h)
+            K = K.numpy()
+            n = int(inp["seq_lens"][b]) // L
+            _, xi, lam = O.build_summaries(K, L, r, n_blocks=n)
+            c_ref = O.build_skew(K, L, xi)
+            for blk in range(n):
+                own = O.block_skew(K[blk * L:(blk + 1) * L], xi_gpu[b, h, blk])
+                assert np.all(np.abs(skew_gpu[b, h, blk] - own) <= 2e-3 * np.maximum(1.0, np.abs(own))), (b, h, blk)
+                for i in range(r):
+                    gaps = [abs(lam[blk, i] - lam[blk, j]) for j in range(r) if j != i]
+                    if lam[blk, i] > 0 and min(gaps) > 0.2 * lam[blk, i] and i < r - 1:
+                        assert abs(skew_gpu[b, h, blk, i] - c_ref[blk, i]) <= 5e-3 * max(1.0, abs(c_ref[blk, i])), (b, h, blk, i)
+                        direct += 1
+    assert direct >= 20
+
+
 def test_context_beyond_the_fused_selection_capacity():
     """4096 blocks per unit: more than the step kernel's selection team holds (2048), so scoring and selection
     take the generic kernels and only attention runs in the persistent kernel; same parity bar."""
