@@ -1,6 +1,6 @@
 """Variants of the descriptor on one shape, through the same kernels: rank 0 (mean-pool score), 4, 6, 8; full key
 space or a query subspace of several widths; bf16 or FP4 factors (the paper's ablation axes: Table "bandwidth",
-Table "quant", the per-layer subspace widths).  For every variant: the record bytes per block and KV head, the
+Table "quant", the per-layer subspace widths, and the appendix's diagonal-skew variant).  For every variant: the record bytes per block and KV head, the
 algorithmic bytes of a decode step, the measured step time on the GPU, and the recall of its selection against the
 exact-mass selector (cobs_exact_select, the paper's OSA reference).  Prints a markdown table.
 
@@ -33,12 +33,12 @@ def algorithmic_bytes(wl: synth.Workload, record: int) -> int:
     return total
 
 
-def time_variant(wl: synth.Workload, steps: int):
+def time_variant(wl: synth.Workload, steps: int, skew: bool = False):
     dev = "cuda"
     inp = synth.generate(wl, dev)
     cfg = B.make_config(wl)
     kv = B.make_kv(inp)
-    summ = B.SummaryBuffers(cfg, dev, inp.get("u_q"))
+    summ = B.SummaryBuffers(cfg, dev, inp.get("u_q"), skew=skew)
     ws = B.alloc_workspace(cfg, dev)
     B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, summ, ws)
     nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
@@ -62,7 +62,7 @@ def time_variant(wl: synth.Workload, steps: int):
     torch.cuda.synchronize()
     us = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)[len(evs) // 2]
     mb, xb, sb = B.cobs_summary_bytes(cfg)
-    record = (mb + xb + sb) // (nb * hkv * wl.max_blocks)
+    record = (mb + xb + sb) // (nb * hkv * wl.max_blocks) + (4 * wl.rank if skew else 0)
     # recall of the estimator's selection against the exact-mass selector (the paper's OSA reference)
     sel_x, cnt_x = torch.zeros_like(sel), torch.zeros_like(cnt)
     B.cobs_exact_select(cfg, inp["q"], kv, sel_x, cnt_x, None, ws)
@@ -91,13 +91,16 @@ def main():
     for s in (42, 56, 71, 85, 108):
         variants.append((f"subspace s={s}, r=4, fp4", base.replace(sub_dim=s, rank=4, summary_dtype="fp4")))
     variants.append(("subspace s=85, r=4, bf16", base.replace(sub_dim=85, rank=4, summary_dtype="bf16")))
+    # the diagonal-skew variant (Appendix, Cheap diagonal skew): r more scalars per block, scored by the generic kernels
+    skewed = [(f"full space, r={rank}, bf16 + skew", base.replace(sub_dim=0, query_model="iid", rank=rank,
+                                                                  summary_dtype="bf16")) for rank in (4, 8)]
     print(f"shape: B={base.batch}, {base.n_q_heads} query / {base.n_kv_heads} KV heads, D={base.head_dim}, "
           f"T={base.seq_len}, L={base.block_size}, k={base.topk}, W={base.window}")
     print("| descriptor | record B / block / KV head | algorithmic MiB / step | step (median, us) | GB/s | "
           "recall of the exact-mass top-k |")
     print("|---|---|---|---|---|---|")
-    for label, wl in variants:
-        record, nbytes, us, recall = time_variant(wl.replace(name=label), args.steps)
+    for label, wl in variants + skewed:
+        record, nbytes, us, recall = time_variant(wl.replace(name=label), args.steps, skew=(label, wl) in skewed)
         print(f"| {label} | {record} | {nbytes / 2**20:.1f} | {us:.1f} | {nbytes / us / 1e3:.0f} | {recall:.3f} |")
 
 
