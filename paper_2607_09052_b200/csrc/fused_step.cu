@@ -1760,7 +1760,7 @@ static cudaError_t launch_fused_t(Params p, int phases, cudaStream_t stream) {
 // Whether the persistent kernel covers this configuration's scoring phase.
 bool fused_score_supported(const Params &p) {
   if (p.skew) return false;                                     // the third-cumulant variant is scored by the generic kernel
-  if (p.NB > kSelThreads * 16 || p.NB % 4 != 0) return false;   // the selection team holds one chunk per thread
+  if (p.NB > kSelThreads * 16 || p.NB % 4 != 0) return false;   // the selection team holds at most 16 blocks per thread
   if (p.summ_dtype == COBS_SUMM_BF16) return p.u_q == nullptr;
   if (p.summ_dtype == COBS_SUMM_FP4_E2M1) {
     if (p.Ds_pad % 32 != 0) return false;
