@@ -761,19 +761,20 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
             }
 #pragma unroll
             for (int k = 0; k < RG; ++k) {
-              float sa = 0.f, sb = 0.f;
-              if (i0 + ((k + gid) & (RG - 1)) < rows) {
-                const int ri = row0 + i0 + ((k + gid) & (RG - 1));
-                if (scale_sz == 4) {
-                  sa = reinterpret_cast<const float *>(sp)[ri];
-                  sb = reinterpret_cast<const float *>(sp)[r + ri];
-                } else {
-                  sa = __half2float(reinterpret_cast<const __half *>(sp)[ri]);
-                  sb = __half2float(reinterpret_cast<const __half *>(sp)[r + ri]);
-                }
+              // scales of this lane's row of the group (clamped like the row itself; a row past the end weighs zero).
+              // The per-head query factors m0, m1 are applied once per chunk, to the sums of squares.
+              const int io = i0 + ((k + gid) & (RG - 1));
+              const int ri = row0 + min(io, rows - 1);
+              float sa, sb;
+              if (scale_sz == 4) {
+                sa = reinterpret_cast<const float *>(sp)[ri];
+                sb = reinterpret_cast<const float *>(sp)[r + ri];
+              } else {
+                sa = __half2float(reinterpret_cast<const __half *>(sp)[ri]);
+                sb = __half2float(reinterpret_cast<const __half *>(sp)[r + ri]);
               }
-              const float d0 = d[k][0] * (sa * m0), d1 = d[k][1] * (sa * m1);
-              const float d2 = d[k][2] * (sb * m0), d3 = d[k][3] * (sb * m1);
+              if (io >= rows) { sa = 0.f; sb = 0.f; }
+              const float d0 = d[k][0] * sa, d1 = d[k][1] * sa, d2 = d[k][2] * sb, d3 = d[k][3] * sb;
               sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
             }
           }
@@ -809,10 +810,12 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
       pend_u = u;
       if (ck * 16 < n_sum) {
         const int bA = ck * 16 + 2 * gid, bB = bA + 1, g0 = 2 * tig, g1 = g0 + 1;
-        const float eA0 = (bA < n_sum) ? ln_l + fA0 + 0.5f * sA0 : -INFINITY;
-        const float eB0 = (bB < n_sum) ? ln_l + fB0 + 0.5f * sB0 : -INFINITY;
-        const float eA1 = (bA < n_sum) ? ln_l + fA1 + 0.5f * sA1 : -INFINITY;
-        const float eB1 = (bB < n_sum) ? ln_l + fB1 + 0.5f * sB1 : -INFINITY;
+        // 1/2 of the sums of squared projections; for FP4 the squares still lack the query's per-head factor
+        const float h0 = FP4 ? 0.5f * m0 * m0 : 0.5f, h1 = FP4 ? 0.5f * m1 * m1 : 0.5f;
+        const float eA0 = (bA < n_sum) ? ln_l + fA0 + h0 * sA0 : -INFINITY;
+        const float eB0 = (bB < n_sum) ? ln_l + fB0 + h0 * sB0 : -INFINITY;
+        const float eA1 = (bA < n_sum) ? ln_l + fA1 + h1 * sA1 : -INFINITY;
+        const float eB1 = (bB < n_sum) ? ln_l + fB1 + h1 * sB1 : -INFINITY;
         // max over the chunk's 16 blocks (over gid), per head
         float mx0 = fmaxf(eA0, eB0), mx1 = fmaxf(eA1, eB1);
 #pragma unroll
