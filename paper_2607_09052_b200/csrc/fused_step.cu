@@ -43,6 +43,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -628,7 +629,6 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     COBS_ACC(1);
 
     const int u = cu, ck = cck, n_sum = cn;
-    const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
     const uint32_t sbase = ring + st * kScoreStageBytes;
     if (ck * 16 < n_sum) {
       if (!mbar_wait(bar0 + st * 8, (phase_bits >> st) & 1u)) {     // bounded: the copies never landed
@@ -642,6 +642,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
         if (cur_b == 0) {
         if (u != cur_u) {
           cur_u = u;
+          const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;      // a division: once per unit, not per chunk
           // ---- query fragments of this unit ------------------------------------------------------------
           const __nv_bfloat16 *qg = p.q + ((size_t)b_idx * p.Hq + h * G) * D;
 #pragma unroll
@@ -759,24 +760,27 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
                 }
               }
             }
+            // scales of this lane's rows of the group (clamped like the rows themselves; a row past the end weighs
+            // zero).  The per-head query factors m0, m1 are applied once per chunk, to the sums of squares.
+            auto accumulate = [&](auto f32) {
 #pragma unroll
-            for (int k = 0; k < RG; ++k) {
-              // scales of this lane's row of the group (clamped like the row itself; a row past the end weighs zero).
-              // The per-head query factors m0, m1 are applied once per chunk, to the sums of squares.
-              const int io = i0 + ((k + gid) & (RG - 1));
-              const int ri = row0 + min(io, rows - 1);
-              float sa, sb;
-              if (scale_sz == 4) {
-                sa = reinterpret_cast<const float *>(sp)[ri];
-                sb = reinterpret_cast<const float *>(sp)[r + ri];
-              } else {
-                sa = __half2float(reinterpret_cast<const __half *>(sp)[ri]);
-                sb = __half2float(reinterpret_cast<const __half *>(sp)[r + ri]);
+              for (int k = 0; k < RG; ++k) {
+                const int io = i0 + ((k + gid) & (RG - 1));
+                const int ri = row0 + min(io, rows - 1);
+                float sa, sb;
+                if (decltype(f32)::value) {
+                  sa = reinterpret_cast<const float *>(sp)[ri];
+                  sb = reinterpret_cast<const float *>(sp)[r + ri];
+                } else {
+                  sa = __half2float(reinterpret_cast<const __half *>(sp)[ri]);
+                  sb = __half2float(reinterpret_cast<const __half *>(sp)[r + ri]);
+                }
+                if (io >= rows) { sa = 0.f; sb = 0.f; }
+                const float d0 = d[k][0] * sa, d1 = d[k][1] * sa, d2 = d[k][2] * sb, d3 = d[k][3] * sb;
+                sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
               }
-              if (io >= rows) { sa = 0.f; sb = 0.f; }
-              const float d0 = d[k][0] * sa, d1 = d[k][1] * sa, d2 = d[k][2] * sb, d3 = d[k][3] * sb;
-              sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
-            }
+            };
+            if (scale_sz == 4) accumulate(std::true_type{}); else accumulate(std::false_type{});
           }
         }
       } else {
