@@ -829,13 +829,13 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
         }
         const float tA0 = __expf(eA0 - mx0), tB0 = __expf(eB0 - mx0), tA1 = __expf(eA1 - mx1), tB1 = __expf(eB1 - mx1);
         float *e0 = p.e + ((size_t)u * G + g0) * NB, *e1 = p.e + ((size_t)u * G + g1) * NB;
-        if (g0 < G) {
-          if (bA < n_sum) __stcg(e0 + bA, tA0);
-          if (bB < n_sum) __stcg(e0 + bB, tB0);
-        }
-        if (g1 < G) {
-          if (bA < n_sum) __stcg(e1 + bA, tA1);
-          if (bB < n_sum) __stcg(e1 + bB, tB1);
+        // blocks bA (even) and bA + 1 are neighbours in memory: one 8-byte store when both exist
+        if (bB < n_sum) {
+          if (g0 < G) __stcg(reinterpret_cast<float2 *>(e0 + bA), make_float2(tA0, tB0));
+          if (g1 < G) __stcg(reinterpret_cast<float2 *>(e1 + bA), make_float2(tA1, tB1));
+        } else if (bA < n_sum) {
+          if (g0 < G) __stcg(e0 + bA, tA0);
+          if (g1 < G) __stcg(e1 + bA, tA1);
         }
         float sm0 = tA0 + tB0, sm1 = tA1 + tB1;
 #pragma unroll
