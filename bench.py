@@ -9,8 +9,11 @@ value is the whole-job achieved HBM bandwidth: algorithmic bytes per step (summa
 summarised block + K and V of the selected and window blocks + q + out) times the number of ranks,
 divided by the step time (CUDA events, max over ranks).  Prints ONE JSON line on rank 0.
 
-With N > 1 (launched by torch.distributed.run) every rank holds its own batch of sequences: the path
-shards over (sequence, KV head) with no collective, so scaling is weak.
+With N > 1 every rank holds its own batch of sequences: the path shards over (sequence, KV head) with no
+collective, so scaling is weak.  `--gpus N` with no rank environment (plain `python bench.py --gpus N`) starts the
+N ranks itself through torch.distributed.run on 127.0.0.1; under torchrun the ranks are taken from the environment.
+The line also carries `other_workloads`: the step time and roofline fraction of the other named configurations
+(fewer steps each), so that one run covers the 32k configurations as well as the 128k one.
 """
 
 from __future__ import annotations
@@ -110,6 +113,145 @@ def dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
 
+def ensure_ranks(args):
+    """Make `--gpus N` mean N ranks.  Under a launcher (WORLD_SIZE set) the environment decides and must agree with
+    the flag; without one and N > 1 this process replaces itself by `python -m torch.distributed.run` with N
+    workers on this node (rendezvous on 127.0.0.1), each of which re-enters this script with its rank set."""
+    if "WORLD_SIZE" in os.environ:
+        world = int(os.environ["WORLD_SIZE"])
+        if args.gpus != world:
+            if int(os.environ.get("RANK", "0")) == 0:
+                sys.stderr.write(f"bench.py: --gpus {args.gpus} but the launcher started {world} ranks; using {world}\n")
+            args.gpus = world
+        return
+    if args.gpus <= 1:
+        return
+    if args.impl == "ours" and not args.launch_selftest:
+        have = torch.cuda.device_count()
+        if args.gpus > have:
+            sys.stderr.write(f"bench.py: --gpus {args.gpus} but this node has {have} CUDA device(s)\n")
+            sys.exit(2)
+    cmd = shard.launcher_command(os.path.abspath(__file__), args.gpus, sys.argv[1:])
+    sys.stdout.flush()
+    os.execvp(cmd[0], cmd)
+
+
+OTHER_WORKLOADS = ["cfg2_32k", "cfg3a_32k_subspace", "cfg3b_32k_k85", "cfg5_64k_g8"]
+
+
+class Measurement:
+    """One workload resident on one GPU: inputs, summaries built by the library, and the timed loops."""
+
+    def __init__(self, B, wl, dev):
+        self.B, self.wl, self.dev = B, wl, dev
+        self.inp = synth.generate(wl, dev)
+        self.cfg = B.make_config(wl)
+        self.kv = B.make_kv(self.inp)
+        self.summ = B.SummaryBuffers(self.cfg, dev, self.inp.get("u_q"))
+        self.ws = B.alloc_workspace(self.cfg, dev)
+        self.stream = torch.cuda.current_stream()
+        nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+        self.out = torch.zeros((nb, hq, D), dtype=torch.float32, device=dev)
+        self.sel = torch.zeros((nb, hkv, wl.topk), dtype=torch.int32, device=dev)
+        self.cnt = torch.zeros((nb, hkv), dtype=torch.int32, device=dev)
+        mb, xb, sb = B.cobs_summary_bytes(self.cfg)
+        self.record = (mb + xb + sb) // (nb * hkv * wl.max_blocks)
+        self.step_bytes = algorithmic_bytes(wl, self.record)
+        self.summary_bytes = sum(hkv * (t // wl.block_size) * self.record for t in wl.lens())
+        # summaries of every block, built by the library (set-up, timed separately)
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(self.stream)
+        B.cobs_build_summaries(self.cfg, self.kv, 0, wl.max_blocks, self.summ, self.ws)
+        ev1.record(self.stream)
+        torch.cuda.synchronize()
+        self.build_ms = ev0.elapsed_time(ev1)
+        self.check("cobs_build_summaries")
+
+    def check(self, where):
+        if self.B.cobs_read_status(self.ws) != 0:
+            raise RuntimeError(f"device status after {where}")
+
+    def step(self):
+        self.B.cobs_decode_step(self.cfg, self.inp["q"], self.kv, self.summ, self.out, None, self.sel, self.cnt, self.ws)
+
+    def timed(self, fn, n, flush):
+        """n calls of fn, each bracketed by CUDA events on the launching stream, an L2 flush (not timed) before
+        each.  Returns the per-call milliseconds."""
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b_ in evs:
+            if flush is not None:
+                flush.zero_()
+            a.record(self.stream)
+            fn()
+            b_.record(self.stream)
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b_) for a, b_ in evs]
+
+    def e2e_seconds(self, n, flush):
+        """n calls of the host-buffer entry point (pinned host q in, host out back, synchronised): wall clock around
+        each call alone; the L2 flush and its synchronise come before the clock starts."""
+        B, wl = self.B, self.wl
+        q_host = self.inp["q"].cpu().pin_memory()
+        out_host = torch.zeros((wl.batch, wl.n_q_heads, wl.head_dim), dtype=torch.float32).pin_memory()
+        for _ in range(2):
+            B.cobs_decode_step_host(self.cfg, q_host, self.kv, self.summ, out_host, None, None, self.ws)
+        total = 0.0
+        for _ in range(n):
+            if flush is not None:
+                flush.zero_()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            B.cobs_decode_step_host(self.cfg, q_host, self.kv, self.summ, out_host, None, None, self.ws)
+            total += time.perf_counter() - t0
+        return total, q_host.numel() * 2, out_host.numel() * 4
+
+
+def measure_other(B, name, dev, flush, peak, steps):
+    """Step time of another named configuration on this GPU (fewer steps; same timing rules)."""
+    wl = synth.named_workloads()[name]
+    m = Measurement(B, wl, dev)
+    for _ in range(5):
+        flush.zero_()
+        m.step()
+    torch.cuda.synchronize()
+    launches0 = B.cobs_kernel_launches()
+    ms = m.timed(m.step, steps, flush)
+    launches = B.cobs_kernel_launches() - launches0
+    m.check("the timed steps")
+    e2e_s, _, _ = m.e2e_seconds(steps, flush)
+    us = statistics.mean(ms) * 1e3
+    gbs = m.step_bytes / (us * 1e-6) / 1e9
+    return {"workload": name, "us_per_step": round(us, 2), "us_per_step_median": round(statistics.median(ms) * 1e3, 2),
+            "algorithmic_bytes_per_step": m.step_bytes, "achieved_gbs": round(gbs, 1), "frac": round(gbs / peak, 4),
+            "e2e_us_per_step": round(e2e_s / steps * 1e6, 2), "kernels_per_step": launches / steps, "steps": steps,
+            "build_summaries_ms": round(m.build_ms, 3),
+            "hbm_time_us_at_peak": round(m.step_bytes / (peak * 1e9) * 1e6, 2)}
+
+
+def run_launch_selftest(args):
+    """The N-rank launch path without a GPU: every rank joins a gloo group, runs a stub step whose duration grows
+    with the rank, and rank 0 prints the line with the real world size and the max-over-ranks time.  What
+    tests/test_shard_gloo.py drives."""
+    import torch.distributed as dist
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    sys.stderr.write(f"bench.py: rank {rank} of {world} up (local rank {local_rank}, launch self-test, no GPU work)\n")
+    wl = shard.rank_workload(synth.named_workloads()["cfg1_tiny"], rank)
+    local_ms = args.steps * (1.0 + rank)                      # the last rank is the slow one
+    total_ms, = shard.job_times([local_ms])
+    if rank == 0:
+        step_bytes = 1000
+        print(json.dumps({"launch_selftest": True, "n_gpus": world, "steps": args.steps, "ms_per_step": total_ms / args.steps,
+                          "value": shard.job_throughput(step_bytes, world, total_ms / args.steps * 1e-3),
+                          "seed_rank0": wl.seed}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_ours(args):
     from paper_2607_09052_b200 import binding as B
     from paper_2607_09052_b200 import build as build_mod
@@ -117,6 +259,8 @@ def run_ours(args):
     rank, local_rank, world = dist_env()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    if local_rank >= torch.cuda.device_count():
+        raise RuntimeError(f"rank {rank}: local rank {local_rank} has no GPU ({torch.cuda.device_count()} visible)")
     torch.cuda.set_device(local_rank)
     if rank == 0:
         build_mod.build()
@@ -124,6 +268,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist.barrier()
+    sys.stderr.write(f"bench.py: rank {rank} of {world} on cuda:{local_rank} ({torch.cuda.get_device_name(local_rank)})\n")
     B.lib()
 
     wl = synth.named_workloads()[args.workload]
@@ -135,35 +280,13 @@ def run_ours(args):
         wl = wl.replace(shuffle_pages=False, name=f"{wl.name}[contiguous pages]")
     wl = shard.rank_workload(wl, rank)                  # every rank draws its own sequences
     dev = torch.device("cuda", local_rank)
-    inp = synth.generate(wl, dev)
-    cfg = B.make_config(wl)
-    kv = B.make_kv(inp)
-    summ = B.SummaryBuffers(cfg, dev, inp.get("u_q"))
-    ws = B.alloc_workspace(cfg, dev)
-    stream = torch.cuda.current_stream()
-
-    # summaries of every block, built by the library (set-up, timed separately)
-    torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, summ, ws)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    build_ms = ev0.elapsed_time(ev1)
-    if B.cobs_read_status(ws) != 0:
-        raise RuntimeError("device status after build_summaries")
-
+    m = Measurement(B, wl, dev)
+    cfg, inp, kv, summ, ws, out, sel, cnt, stream = m.cfg, m.inp, m.kv, m.summ, m.ws, m.out, m.sel, m.cnt, m.stream
     nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
-    out = torch.zeros((nb, hq, D), dtype=torch.float32, device=dev)
-    sel = torch.zeros((nb, hkv, wl.topk), dtype=torch.int32, device=dev)
-    cnt = torch.zeros((nb, hkv), dtype=torch.int32, device=dev)
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    mb, xb, sb = B.cobs_summary_bytes(cfg)
-    record = (mb + xb + sb) // (nb * hkv * wl.max_blocks)
-    step_bytes = algorithmic_bytes(wl, record)
-
-    def step():
-        B.cobs_decode_step(cfg, inp["q"], kv, summ, out, None, sel, cnt, ws)
+    record, step_bytes, build_ms = m.record, m.step_bytes, m.build_ms
+    flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush = None if args.no_l2_flush else flush_buf
+    step = m.step
 
     def barrier():
         torch.cuda.synchronize()
@@ -176,7 +299,7 @@ def run_ours(args):
     t_warm = time.perf_counter()
     n_warm = 0
     while n_warm < args.warmup or time.perf_counter() - t_warm < args.clock_warm_s:   # >= W steps, and long enough for clock samples
-        if not args.no_l2_flush:
+        if flush is not None:
             flush.zero_()
         step()
         n_warm += 1
@@ -185,60 +308,28 @@ def run_ours(args):
     barrier()
 
     # ---- timed region: exactly K steps, an L2 flush (not timed) before each ----------------------------
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     launches0 = B.cobs_kernel_launches()
     t_wall0 = time.perf_counter()
-    for i in range(args.steps):
-        if not args.no_l2_flush:
-            flush.zero_()
-        starts[i].record(stream)
-        step()
-        ends[i].record(stream)
+    step_ms = m.timed(step, args.steps, flush)
     barrier()
     wall_s = time.perf_counter() - t_wall0
     launches = B.cobs_kernel_launches() - launches0
     clocks = sampler.stop() if sampler else None
-    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
     total_ms = sum(step_ms)
-    if B.cobs_read_status(ws) != 0:
-        raise RuntimeError("device status after the timed steps")
+    m.check("the timed steps")
 
     # ---- the two halves of the step through their own entry points (context for the roofline line) ----
-    def time_call(fn, n):
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
-        for a, b_ in evs:
-            flush.zero_()
-            a.record(stream)
-            fn()
-            b_.record(stream)
-        torch.cuda.synchronize()
-        return sum(a.elapsed_time(b_) for a, b_ in evs) / n
-
     n_sub = max(3, min(args.steps, 20))
-    score_ms = time_call(lambda: B.cobs_score_select(cfg, inp["q"], summ, inp["seq_lens"], sel, cnt, None, ws), n_sub)
-    attend_ms = time_call(lambda: B.cobs_sparse_decode(cfg, inp["q"], kv, sel, cnt, out, None, ws), n_sub)
-    summary_bytes = sum(hkv * (t // wl.block_size) * record for t in wl.lens())
+    score_ms = statistics.mean(m.timed(lambda: B.cobs_score_select(cfg, inp["q"], summ, inp["seq_lens"], sel, cnt, None, ws),
+                                       n_sub, flush_buf))
+    attend_ms = statistics.mean(m.timed(lambda: B.cobs_sparse_decode(cfg, inp["q"], kv, sel, cnt, out, None, ws),
+                                        n_sub, flush_buf))
+    summary_bytes = m.summary_bytes
     kv_bytes = step_bytes - summary_bytes
 
     # ---- end to end through the host-buffer entry point ------------------------------------------------
-    q_host = inp["q"].cpu().pin_memory()
-    out_host = torch.zeros((nb, hq, D), dtype=torch.float32).pin_memory()
-    for _ in range(2):
-        B.cobs_decode_step_host(cfg, q_host, kv, summ, out_host, None, None, ws)
     barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        flush.zero_()
-        torch.cuda.synchronize()
-        B.cobs_decode_step_host(cfg, q_host, kv, summ, out_host, None, None, ws)
-    e2e_s = time.perf_counter() - t0
-    # the flush and its synchronise are inside this wall-clock loop; time them alone and take them out
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        flush.zero_()
-        torch.cuda.synchronize()
-    e2e_s = max(e2e_s - (time.perf_counter() - t0), 1e-9)
+    e2e_s, h2d_bytes, d2h_bytes = m.e2e_seconds(args.steps, flush_buf)
 
     # ---- optional: consecutive decode steps (append a token, rebuild a block's summary when it fills, step) ----
     loop_info = None
@@ -260,8 +351,7 @@ def run_ours(args):
             loop.step(q_i, k_i, v_i, out, None, sel, cnt)
         ev_b.record(stream)
         torch.cuda.synchronize()
-        if B.cobs_read_status(ws) != 0:
-            raise RuntimeError("device status after the decode loop")
+        m.check("the decode loop")
         loop_info = {"steps": n_loop, "start_len": start_len, "rebuilds": loop.rebuilds,
                      "us_per_step_amortised": round(ev_a.elapsed_time(ev_b) * 1e3 / n_loop, 2),
                      "note": "append + summary rebuild of the block that filled (one launch per block boundary, all "
@@ -284,6 +374,7 @@ def run_ours(args):
         "metric": "fused COBS decode step: achieved HBM GB/s (algorithmic bytes per step / step time)",
         "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": round(ms_per_step, 6), "us_per_step": round(ms_per_step * 1e3, 3),
+        "us_per_step_median": round(statistics.median(step_ms) * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "batch_per_gpu": nb, "global_batch": nb * world, "context": wl.seq_len,
                    "n_q_heads": hq, "n_kv_heads": hkv, "head_dim": D, "block_size": wl.block_size,
@@ -306,7 +397,9 @@ def run_ours(args):
                              f"capture summarised under profiles/ (null when not captured for this workload)"},
         "e2e": {"value": round(world * step_bytes / (e2e_s / args.steps) / 1e9, 2), "unit": "GB/s",
                 "us_per_step": round(e2e_s / args.steps * 1e6, 2),
-                "h2d_bytes_per_step": q_host.numel() * 2, "d2h_bytes_per_step": out_host.numel() * 4},
+                "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes,
+                "note": "cobs_decode_step_host: pinned host q copied in, step, output written to pinned host memory, "
+                        "stream synchronised; wall clock around each call alone"},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "build_summaries_ms": round(build_ms, 3),
@@ -314,6 +407,10 @@ def run_ours(args):
     }
     if loop_info:
         line["decode_loop"] = loop_info
+    if world == 1 and not args.no_other_workloads and args.workload == DEFAULT_WORKLOAD and not (args.batch or args.seq_len):
+        del m, step, inp, kv, summ, ws, out, sel, cnt
+        torch.cuda.empty_cache()
+        line["other_workloads"] = [measure_other(B, name, dev, flush_buf, peak, args.other_steps) for name in OTHER_WORKLOADS]
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl, record, budget_s=20.0)
     print(json.dumps(line), flush=True)
@@ -429,9 +526,17 @@ def main():
                          "report the amortised time per step")
     ap.add_argument("--clock-warm-s", type=float, default=0.6,
                     help="keep warming up at least this long so that the clock sampler has samples")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the other named configurations (the `other_workloads` list of the line)")
+    ap.add_argument("--other-steps", type=int, default=20, help="timed steps per other configuration")
+    ap.add_argument("--launch-selftest", action="store_true",
+                    help="no GPU work: bring the N ranks up on gloo, run a stub step, print the line (tests the launch path)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    ensure_ranks(args)
+    if args.launch_selftest:
+        run_launch_selftest(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

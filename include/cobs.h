@@ -62,6 +62,8 @@ typedef enum { COBS_SCALE_FP32 = 0, COBS_SCALE_FP16 = 1 } cobs_scale_dtype;
 
 #define COBS_MAX_TOPK 128
 #define COBS_MAX_RANK 16
+#define COBS_MAX_BLOCKS 57344       /* largest max_blocks (3.67 M tokens of context at L = 64) */
+#define COBS_MAX_UNITS 65535        /* largest batch * n_kv_heads */
 
 /* Problem statement: shapes and method parameters (paper: Background, Notation; Method). */
 typedef struct {
@@ -77,8 +79,8 @@ typedef struct {
   int32_t window;             /* local window in tokens, >= 1 */
   int32_t summary_dtype;      /* cobs_summary_dtype */
   int32_t scale_dtype;        /* cobs_scale_dtype; read only when summary_dtype == COBS_SUMM_FP4_E2M1 */
-  int32_t max_blocks;         /* NB: block capacity per sequence = stride of the summary arrays */
-  int32_t max_pages_per_seq;  /* row stride of page_table */
+  int32_t max_blocks;         /* NB: block capacity per sequence = stride of the summary arrays; <= COBS_MAX_BLOCKS */
+  int32_t max_pages_per_seq;  /* row stride of page_table; max_pages_per_seq * P >= NB * L */
 } cobs_config;
 
 /* Paged bf16 KV cache. */
@@ -86,7 +88,9 @@ typedef struct {
   const void *k_pages;        /* [n_pages][Hkv][P][D] bf16 */
   const void *v_pages;        /* [n_pages][Hkv][P][D] bf16 */
   const int32_t *page_table;  /* [B][max_pages_per_seq]: page id of the i-th page of a sequence */
-  const int32_t *seq_lens;    /* [B]: tokens in the cache, the current one included; 1 <= T <= NB*L + L - 1 */
+  const int32_t *seq_lens;    /* [B]: tokens in the cache, the current one included; 1 <= T <= min(NB*L + L - 1,
+                                 max_pages_per_seq * P).  Tokens beyond the page-table row are not read: they are
+                                 skipped and COBS_ERR_BOUNDS is left in the status word */
   int64_t n_pages;            /* page ids are checked against this */
 } cobs_kv;
 
@@ -177,6 +181,16 @@ int32_t cobs_append_token(const cobs_config *cfg, const void *k_new, const void 
  */
 int32_t cobs_quantise_xi(const cobs_config *cfg, const float *xi_fp32, int64_t n_vectors, void *codes, void *scale,
                          void *stream);
+
+/*
+ * Test hook for the E2M1 rounding rule (Method, Quantization names the format; the rounding is the format's
+ * round-to-nearest-even): codes[i] = the code the GPU's own conversion instruction (cvt.rn.satfinite.e2m1x2.f32)
+ * gives x[i], one byte per value (bit 3 sign, bits 2..0 magnitude index).  x device fp32 [n], codes device bytes
+ * [n]; n <= 2^31.  cobs_quantise_xi does not use that instruction (it must divide by the scale in fp32 and keep
+ * the sign of a value that rounds to zero, both by its own rule); the parity tests compare the two on a dense grid.
+ * Nothing on the decode path calls this.
+ */
+int32_t cobs_hw_e2m1_codes(const float *x, int64_t n, uint8_t *codes, void *stream);
 
 /*
  * (b) + (c) Score every summarised block and select (Eq. trunc, Eq. gram, Eq. gqa-secondorder).

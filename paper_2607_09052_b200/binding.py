@@ -12,8 +12,6 @@ from typing import Optional
 
 import torch
 
-from .synth import Workload
-
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcobs.so")
 
@@ -24,7 +22,7 @@ EXPORTS = [
     "cobs_status_string", "cobs_padded_sub_dim", "cobs_summary_bytes", "cobs_workspace_bytes", "cobs_reset_status",
     "cobs_read_status", "cobs_build_summaries", "cobs_quantise_xi", "cobs_score_select", "cobs_sparse_decode",
     "cobs_decode_step", "cobs_decode_step_host", "cobs_kernel_launches", "cobs_tcgen05_launches", "cobs_sparse_decode_static", "cobs_append_token", "cobs_exact_select",
-    "cobs_adaptive_trim",
+    "cobs_adaptive_trim", "cobs_hw_e2m1_codes",
 ]
 
 
@@ -98,7 +96,10 @@ def _stream(stream) -> C.c_void_p:
     return C.c_void_p(stream.cuda_stream)
 
 
-def make_config(wl: Workload) -> Config:
+def make_config(wl) -> Config:
+    """The library's configuration struct from any object that names a decode problem by the attributes batch,
+    n_q_heads, n_kv_heads, head_dim, block_size, page_size, rank, sub_dim, topk, window, summary_dtype
+    ("fp32" | "bf16" | "fp4"), scale_dtype ("fp32" | "fp16"), max_blocks and max_pages_per_seq."""
     return Config(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.block_size, wl.page_size, wl.rank, wl.sub_dim,
                   wl.topk, wl.window, SUMM_DTYPES[wl.summary_dtype], SCALE_DTYPES[wl.scale_dtype], wl.max_blocks,
                   wl.max_pages_per_seq)
@@ -188,6 +189,12 @@ def cobs_quantise_xi(cfg: Config, xi_fp32: torch.Tensor, codes: torch.Tensor, sc
     n_vectors = xi_fp32.shape[0]
     _check(lib().cobs_quantise_xi(C.byref(cfg), _ptr(xi_fp32), C.c_int64(n_vectors), _ptr(codes), _ptr(scale),
                                   _stream(stream)), "cobs_quantise_xi")
+
+
+def cobs_hw_e2m1_codes(x: torch.Tensor, codes: torch.Tensor, stream=None):
+    """codes[i] = the E2M1 code the GPU's own conversion instruction gives x[i] (test hook for the rounding rule)."""
+    assert x.dtype == torch.float32 and codes.dtype == torch.uint8 and x.numel() == codes.numel()
+    _check(lib().cobs_hw_e2m1_codes(_ptr(x), C.c_int64(x.numel()), _ptr(codes), _stream(stream)), "cobs_hw_e2m1_codes")
 
 
 def cobs_score_select(cfg: Config, q: torch.Tensor, summ: SummaryBuffers, seq_lens: torch.Tensor,

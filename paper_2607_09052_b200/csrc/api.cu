@@ -58,12 +58,16 @@ static int32_t validate_config(const cobs_config *c) {
   if (c->summary_dtype < COBS_SUMM_FP32 || c->summary_dtype > COBS_SUMM_FP4_E2M1) return COBS_ERR_INVALID_ARG;
   if (c->summary_dtype == COBS_SUMM_FP4_E2M1 && c->scale_dtype != COBS_SCALE_FP32 && c->scale_dtype != COBS_SCALE_FP16)
     return COBS_ERR_INVALID_ARG;
-  if (c->max_blocks < 1 || c->max_blocks > (1 << 20)) return COBS_ERR_INVALID_ARG;
+  if (c->max_blocks < 1) return COBS_ERR_INVALID_ARG;
+  // the generic selection kernel keeps a unit's scores in shared memory (4 bytes per block, 227 KB at most)
+  if (c->max_blocks > COBS_MAX_BLOCKS) return COBS_ERR_UNSUPPORTED;
   if (c->max_pages_per_seq < 1) return COBS_ERR_INVALID_ARG;
-  // the page table must cover every token a sequence may hold: NB * L + L - 1 at most
+  // the page table must cover every full block (NB * L tokens); a sequence longer than max_pages_per_seq * P
+  // is caught on the device (COBS_ERR_BOUNDS, the tokens beyond the table are skipped)
   if ((long long)c->max_pages_per_seq * c->page_size < (long long)c->max_blocks * c->block_size) return COBS_ERR_INVALID_ARG;
   // an attention slice holds at most kItemGroups 16-token groups and a unit at most kMaxSplits slices
   if ((long long)max_items(c) * (c->block_size / 16) > (long long)kItemGroups * kMaxSplits) return COBS_ERR_UNSUPPORTED;
+  // units index grid.y of the generic scoring kernel (65535 at most) and the workspace's counters
   if ((long long)c->batch * c->n_kv_heads > kMaxUnits) return COBS_ERR_UNSUPPORTED;
   // chunk and item indices are 32-bit
   if ((long long)c->batch * c->n_kv_heads * ((c->max_blocks + 15) / 16) > 0x3fffffffLL) return COBS_ERR_UNSUPPORTED;
@@ -278,6 +282,8 @@ int32_t cobs_build_summaries(const cobs_config *cfg, const cobs_kv *kv, int32_t 
   if ((st = set_kv(p, kv)) != COBS_OK) return st;
   if ((st = set_summaries(p, cfg, out)) != COBS_OK) return st;
   if (build_smem_bytes(p) > 227 * 1024) return COBS_ERR_UNSUPPORTED;
+  // one CTA per (sequence, KV head, block of the range): the grid's x extent is 2^31 - 1 at most
+  if ((long long)p.B * p.Hkv * (block_end - block_begin) > 0x7fffffffLL) return COBS_ERR_UNSUPPORTED;
   return cuda_status(launch_build(p, block_begin, block_end, static_cast<cudaStream_t>(stream)));
 }
 

@@ -12,7 +12,7 @@ namespace cobs {
 
 constexpr int kStatusBytes = 256;          // status word lives in the first 256 bytes of the workspace
 constexpr int kMaxSplits = 64;             // upper bound on split-KV partials per (sequence, KV head)
-constexpr int kMaxUnits = 65536;           // (sequence, KV head) units a workspace has counters for
+constexpr int kMaxUnits = 65535;           // (sequence, KV head) units a workspace has counters for
 constexpr int kCtlBytes = kStatusBytes + 3 * kMaxUnits * 4;   // status word + counters, zeroed by cobs_reset_status
 
 // Everything a kernel needs, passed by value.

@@ -70,7 +70,8 @@ __global__ void __launch_bounds__(kEWarps * 32) exact_mass_kernel(Params p) {
     auto issue = [&](int g, int st) {
       if (g < gpb) {
         const int tok0 = blk * L + g * 16;
-        const int pg = p.page_table[(size_t)b_idx * p.mpp + tok0 / P];
+        const int pslot = tok0 / P;                 // < mpp for every full block (mpp * P >= NB * L); checked all the same
+        const int pg = (pslot < p.mpp) ? p.page_table[(size_t)b_idx * p.mpp + pslot] : -1;
         if (pg < 0 || pg >= p.n_pages) report(p.status, COBS_ERR_BOUNDS);
         else {
           const uint4 *ks = kbase + ((((size_t)pg * p.Hkv + h) * P + (tok0 % P)) * D) / 8;

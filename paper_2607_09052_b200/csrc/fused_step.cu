@@ -223,9 +223,9 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
   static_assert(kSelWarps == 4, "one 16-byte read takes the four warps' words");
   constexpr int NQ = BPT / 4;                    // groups of four blocks of a thread
   constexpr int GB = (BPT == 16) ? 4 : 8;        // heads whose t values are in registers at a time
-  constexpr int CW = (BPT == 16) ? 2 : 1;        // words the three counts of a bisection round are packed in
+  constexpr int CW = (BPT == 4) ? 1 : 2;         // words the three counts of a bisection round are packed in
   __shared__ float s_m[8][kSelWarps], s_s[8][kSelWarps];
-  __shared__ __align__(16) int s_cnt[2][2][kSelWarps];
+  __shared__ __align__(16) uint32_t s_cnt[2][2][kSelWarps];
   __shared__ int s_scan[kSelWarps];
   const int warp = tid >> 5, lane = tid & 31;
   const int G = p.G, NB = p.NB, cpu = (NB + 15) / 16, n_chunks = (n_sum + 15) / 16;
@@ -352,20 +352,22 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
   }
   // k-th largest key by bisection on its bits (scores are >= 0, so their bit patterns order like integers):
   // theta = the largest T with #(key >= T) >= k.  Bit 30 alone, then two bits per round: three trial values, whose
-  // counts travel packed (11 bits each in one word while a team holds at most 1024 keys, else 16 bits each in two
-  // words): per round one or two warp reductions, one shared store per warp, one barrier, one 16-byte read per word.
+  // counts travel packed as unsigned fields (11, 11 and 10 bits of one word while a team holds at most 512 keys - no
+  // field can reach its width - else 16 bits each in two words): per round one or two warp reductions, one shared
+  // store per warp, one barrier, one 16-byte read per word.
   constexpr int SH = (CW == 1) ? 11 : 16, SH2 = (CW == 1) ? 22 : 0;
+  static_assert(CW == 2 || kSelThreads * BPT < (1 << 10), "a packed count would overflow its field");
   int par = 0;
-  auto cta_sum = [&](int c0, int c1, int &n0, int &n1) {
+  auto cta_sum = [&](uint32_t c0, uint32_t c1, uint32_t &n0, uint32_t &n1) {
     c0 = __reduce_add_sync(0xffffffffu, c0);
     if (CW == 2) c1 = __reduce_add_sync(0xffffffffu, c1);
     if (lane == 0) { s_cnt[par][0][warp] = c0; if (CW == 2) s_cnt[par][1][warp] = c1; }
     team_sync();
-    const int4 v = *reinterpret_cast<const int4 *>(&s_cnt[par][0][0]);
+    const uint4 v = *reinterpret_cast<const uint4 *>(&s_cnt[par][0][0]);
     n0 = v.x + v.y + v.z + v.w;
     n1 = 0;
     if (CW == 2) {
-      const int4 w = *reinterpret_cast<const int4 *>(&s_cnt[par][1][0]);
+      const uint4 w = *reinterpret_cast<const uint4 *>(&s_cnt[par][1][0]);
       n1 = w.x + w.y + w.z + w.w;
     }
     par ^= 1;
@@ -373,24 +375,25 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
   uint32_t theta = 0u;
   {
     const uint32_t t = 1u << 30;
-    int c = 0, n0, n1;
+    uint32_t c = 0, n0, n1;
 #pragma unroll
     for (int j = 0; j < BPT; ++j) c += (keys[j] >= t);
-    cta_sum(c, 0, n0, n1);
-    if (n0 >= k) theta = t;
+    cta_sum(c, 0u, n0, n1);
+    if (n0 >= (uint32_t)k) theta = t;
   }
   for (int bit = 29; bit >= 1; bit -= 2) {
     const uint32_t ta = theta | (3u << (bit - 1)), tb = theta | (2u << (bit - 1)), tc = theta | (1u << (bit - 1));
-    int c0 = 0, c1 = 0, n0, n1;
+    uint32_t c0 = 0, c1 = 0, n0, n1;
 #pragma unroll
     for (int j = 0; j < BPT; ++j) {
-      c0 += (keys[j] >= ta ? 1 : 0) + (keys[j] >= tb ? (1 << SH) : 0);
-      if (CW == 1) c0 += (keys[j] >= tc ? (1 << SH2) : 0);
-      else c1 += (keys[j] >= tc ? 1 : 0);
+      c0 += (keys[j] >= ta ? 1u : 0u) + (keys[j] >= tb ? (1u << SH) : 0u);
+      if (CW == 1) c0 += (keys[j] >= tc ? (1u << SH2) : 0u);
+      else c1 += (keys[j] >= tc ? 1u : 0u);
     }
     cta_sum(c0, c1, n0, n1);
-    const int na = n0 & ((1 << SH) - 1), nb = (n0 >> SH) & ((1 << SH) - 1), nc = (CW == 1) ? (n0 >> SH2) : n1;
-    if (na >= k) theta = ta; else if (nb >= k) theta = tb; else if (nc >= k) theta = tc;
+    const uint32_t ku = (uint32_t)k;
+    const uint32_t na = n0 & ((1u << SH) - 1), nb = (n0 >> SH) & ((1u << SH) - 1), nc = (CW == 1) ? (n0 >> SH2) : n1;
+    if (na >= ku) theta = ta; else if (nb >= ku) theta = tb; else if (nc >= ku) theta = tc;
   }
   COBS_SEL_STAMP(4);
   // keep every key above theta and the lowest-index `need_eq` keys equal to it, in index order: one scan of the
@@ -410,7 +413,7 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
   int base = 0, total = 0;
 #pragma unroll
   for (int q = 0; q < kSelWarps; ++q) { const int t = s_scan[q]; total += t; base += (q < warp) ? t : 0; }
-  const int need_eq = k - (total >> 16);
+  const int need_eq = max(k - (total >> 16), 0);
   const int excl = base + inc - v;
   int eq_rank = excl & 0xffff;
   int pos = (excl >> 16) + min(eq_rank, need_eq);
@@ -420,7 +423,7 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
       bool keep = false;
       if (keys[j] > theta) keep = true;
       else if (keys[j] == theta) { keep = eq_rank < need_eq; ++eq_rank; }
-      if (keep && pos < k) out[pos++] = b0 + j;
+      if (keep && pos >= 0 && pos < k) out[pos++] = b0 + j;
     }
   }
   COBS_SEL_STAMP(5);
@@ -1056,7 +1059,8 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
       int first = -1;
       uint32_t off = 0;
       if (good && tok0 < T) {
-        const int pg = p.page_table[(size_t)b_idx * p.mpp + tok0 / P];
+        const int pslot = tok0 / P;                                  // a length beyond the page-table row is not followed
+        const int pg = (pslot < p.mpp) ? p.page_table[(size_t)b_idx * p.mpp + pslot] : -1;
         if (pg < 0 || pg >= p.n_pages) report(p.status, COBS_ERR_BOUNDS);
         else { first = tok0; off = (uint32_t)(((((size_t)pg * p.Hkv + h) * P + (tok0 % P)) * D) / 8); }
       }

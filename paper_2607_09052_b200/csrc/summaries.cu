@@ -414,4 +414,25 @@ cudaError_t launch_quantise(const float *xi, long long n_vectors, int Ds, int Ds
   return cudaGetLastError();
 }
 
+// The GPU's own float -> E2M1 conversion instruction, one code per input value: what the threshold chain of
+// e2m1_encode is checked against (a test hook; nothing on the path calls it).
+__global__ void hw_e2m1_kernel(const float *x, long long n, uint8_t *codes) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t r;
+  // the instruction packs two codes in a byte; the partner value is +0 (code 0), so the OR of the byte's two
+  // nibbles is the code of x[i] whichever nibble the instruction puts it in
+  asm("{\n .reg .b8 t;\n cvt.rn.satfinite.e2m1x2.f32 t, %1, %2;\n cvt.u32.u8 %0, t;\n}\n" : "=r"(r) : "f"(x[i]), "f"(0.0f));
+  codes[i] = (uint8_t)(((r >> 4) | r) & 15u);
+}
+
 }  // namespace cobs
+
+extern "C" int32_t cobs_hw_e2m1_codes(const float *x, int64_t n, uint8_t *codes, void *stream) {
+  if (!x || !codes || n < 0) return COBS_ERR_INVALID_ARG;
+  if (n == 0) return COBS_OK;
+  if (n > ((int64_t)1 << 31)) return COBS_ERR_UNSUPPORTED;
+  cobs::hw_e2m1_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(x, n, codes);
+  cobs::count_launch();
+  return cudaGetLastError() == cudaSuccess ? COBS_OK : COBS_ERR_CUDA;
+}

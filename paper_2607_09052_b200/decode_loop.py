@@ -12,12 +12,11 @@ from typing import Optional
 import torch
 
 from . import binding as B
-from .synth import Workload
 
 
 class DecodeLoop:
-    def __init__(self, wl: Workload, inputs, summ: Optional[B.SummaryBuffers] = None, ws: Optional[torch.Tensor] = None):
-        """`inputs`: device tensors k_pages, v_pages, page_table, seq_lens (and u_q for a subspace descriptor) of a
+    def __init__(self, wl, inputs, summ: Optional[B.SummaryBuffers] = None, ws: Optional[torch.Tensor] = None):
+        """`wl`: the decode problem (any object binding.make_config accepts).  `inputs`: device tensors k_pages, v_pages, page_table, seq_lens (and u_q for a subspace descriptor) of a
         cache with room for the tokens to come: max_blocks * block_size tokens per sequence at most."""
         self.wl = wl
         self.inputs = inputs

@@ -7,13 +7,14 @@ the benchmark: the step time of the job is the slowest rank's.
 
 from __future__ import annotations
 
+import socket
+import sys
+
 import torch
 import torch.distributed as dist
 
-from .synth import Workload
 
-
-def rank_workload(wl: Workload, rank: int) -> Workload:
+def rank_workload(wl, rank: int):
     """The workload rank `rank` draws: same shapes, its own sequences (seed offset by the rank)."""
     return wl.replace(seed=wl.seed + 1000 * rank)
 
@@ -29,3 +30,16 @@ def job_times(local_values, device="cpu"):
 def job_throughput(bytes_per_rank_step: int, world: int, max_step_seconds: float) -> float:
     """Whole-job GB/s: all ranks' bytes over the slowest rank's step time."""
     return world * bytes_per_rank_step / max_step_seconds / 1e9
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launcher_command(script: str, n_ranks: int, argv, port: int = 0):
+    """The command that starts `n_ranks` ranks of `script` on this node: torch.distributed.run, one process per
+    rank (per GPU), rendezvous on 127.0.0.1 (a container's hostname may not resolve)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port or free_port()), script, *argv]
