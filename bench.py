@@ -67,6 +67,27 @@ def read_peaks():
     return 6650.0, "fallback"
 
 
+class L2Flush:
+    """Between timed steps: write a buffer twice the size of L2.  That alone leaves L2 full of DIRTY lines, whose
+    write-back then competes with the next step's reads for HBM (up to 126 MB of extra DRAM writes inside the timed
+    region: an artefact of the flush, not of the workload), so the default mode reads a second buffer of the same
+    size afterwards: L2 then holds clean lines of an unrelated buffer.  Mode "write" is the plain write."""
+
+    def __init__(self, dev, mode="write+read"):
+        self.mode = mode
+        self.buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+        self.src = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=dev) if mode == "write+read" else None
+
+    def zero_(self):
+        self.buf.zero_()
+        if self.src is not None:
+            torch.max(self.src)
+
+    def describe(self):
+        what = "write" if self.src is None else "write, then read of a second buffer of that size (leaves L2 clean)"
+        return f"{L2_FLUSH_BYTES >> 20} MiB {what} between timed steps (outside the events)"
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples while the timed region runs."""
 
@@ -229,6 +250,82 @@ def measure_other(B, name, dev, flush, peak, steps):
             "hbm_time_us_at_peak": round(m.step_bytes / (peak * 1e9) * 1e6, 2)}
 
 
+def run_phase_times(args):
+    """Where the time of one step goes, from the library build that carries timing code (libcobs_timing.so):
+    per-warp global-timer stamps at the phase boundaries, clock cycles per category inside the phases, and per
+    unit the moments its scores were complete and its selection was published.  One JSON line; times in
+    microseconds from the earliest warp's start.  Numbers of this build are not benchmark values."""
+    import ctypes as C
+    import numpy as np
+    from paper_2607_09052_b200 import binding as B
+    from paper_2607_09052_b200 import build as build_mod
+    B.use_library(build_mod.build(timing=True))
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    wl = synth.named_workloads()[args.workload]
+    if args.batch:
+        wl = wl.replace(batch=args.batch)
+    if args.seq_len:
+        wl = wl.replace(seq_len=args.seq_len)
+    m = Measurement(B, wl, dev)
+    flush = L2Flush(dev, args.flush_mode)
+    score_only = args.phase_times == "score"
+    def step():
+        if score_only:
+            B.cobs_score_select(m.cfg, m.inp["q"], m.summ, m.inp["seq_lens"], m.sel, m.cnt, None, m.ws)
+        else:
+            m.step()
+    for _ in range(5):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    acc = (C.c_ulonglong * (8 * 4096))()
+    B.lib().cobs_debug_acc(acc, 1)                          # clear the accumulators
+    flush.zero_()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(m.stream)
+    step()
+    ev1.record(m.stream)
+    torch.cuda.synchronize()
+    buf = (C.c_ulonglong * (4 * 4096))()
+    assert B.lib().cobs_debug_times(buf) == 0 and B.lib().cobs_debug_acc(acc, 1) == 0
+    t = np.frombuffer(buf, dtype=np.uint64).reshape(4, 4096).astype(np.int64)
+    n = int((t[0] > 0).sum())
+    t = t[:, :n]
+    t0 = int(t[0].min())
+    raw = np.frombuffer(acc, dtype=np.uint64).reshape(8, 4096).astype(np.int64)
+    mhz = 1965.0
+
+    def stats(x):
+        return {k: round(float(v), 2) for k, v in zip(("min", "p10", "p50", "p90", "max"),
+                                                      [x.min(), *np.percentile(x, [10, 50, 90]), x.max()])}
+    out = {"phase_times": True, "workload": wl.name, "mode": args.phase_times, "streaming_warps": n,
+           "step_us_this_build": round(ev0.elapsed_time(ev1) * 1e3, 2),
+           "warp_stamps_us": {name: stats((t[k] - t0) / 1e3) for k, name in
+                              enumerate(["start", "scoring_done", "attention_start", "attention_done"])}}
+    sc = raw[:, 1200:1200 + n].astype(np.float64) / mhz
+    busy = sc.sum(0) > 0.5
+    names_s = ["next position", "after issue", "wait for copies", "arithmetic", "epilogue", "issue copies", "seek", "fence + count"]
+    out["scoring_us_per_working_warp"] = {nm: round(float(sc[k][busy].mean()), 2) for k, nm in enumerate(names_s)}
+    out["scoring_working_warps"] = int(busy.sum())
+    if not score_only:
+        at = raw[:, :n].astype(np.float64) / mhz
+        names_a = ["draw item", "item set-up", "wait for selection", "group table + query", "stream loop", "write partial", "close + merge"]
+        out["attention_us_per_warp"] = {nm: round(float(at[k].mean()), 2) for k, nm in enumerate(names_a)}
+        late = np.argsort(t[3])[-8:]
+        out["latest_warps"] = [{"warp": int(w), "attention_start": round(float((t[2][w] - t0) / 1e3), 1),
+                                "attention_done": round(float((t[3][w] - t0) / 1e3), 1),
+                                **{nm: round(float(at[k][w]), 1) for k, nm in enumerate(names_a)}} for w in late]
+    nu = wl.batch * wl.n_kv_heads
+    st = [(raw[k, 3000:3000 + min(nu, 1024)] - t0) / 1e3 for k in (0, 2, 3, 4, 5, 1)]
+    out["selection_us"] = {"unit_scored_at": stats(st[0]), "unit_ready_at": stats(st[5]),
+                           "duration": stats(st[5] - st[0]),
+                           "parts_mean": {nm: round(float((st[i + 1] - st[i]).mean()), 2) for i, nm in
+                                          enumerate(["loads + lse", "scores", "bisection", "compaction", "fence + flag"])}}
+    out["status"] = B.cobs_read_status(m.ws)
+    print(json.dumps(out), flush=True)
+
+
 def run_launch_selftest(args):
     """The N-rank launch path without a GPU: every rank joins a gloo group, runs a stub step whose duration grows
     with the rank, and rank 0 prints the line with the real world size and the max-over-ranks time.  What
@@ -284,7 +381,7 @@ def run_ours(args):
     cfg, inp, kv, summ, ws, out, sel, cnt, stream = m.cfg, m.inp, m.kv, m.summ, m.ws, m.out, m.sel, m.cnt, m.stream
     nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
     record, step_bytes, build_ms = m.record, m.step_bytes, m.build_ms
-    flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_buf = L2Flush(dev, args.flush_mode)
     flush = None if args.no_l2_flush else flush_buf
     step = m.step
 
@@ -381,8 +478,7 @@ def run_ours(args):
                    "page_size": wl.page_size, "topk": wl.topk, "window": wl.window, "rank": wl.rank,
                    "sub_dim": wl.sub_dim, "summary_dtype": wl.summary_dtype, "scale_dtype": wl.scale_dtype,
                    "record_bytes": record, "algorithmic_bytes_per_step": step_bytes,
-                   "l2": ("no flush: " if args.no_l2_flush else
-                          f"{L2_FLUSH_BYTES >> 20} MiB write between timed steps (outside the events); ") +
+                   "l2": ("no flush (the step's own traffic exceeds L2); " if args.no_l2_flush else flush_buf.describe() + "; ") +
                          f"step traffic {step_bytes / 2**20:.1f} MiB",
                    "sharding": "independent sequences per rank, no collective"},
         "frac_of_measured_peak": round(value / (world * peak), 4), "peak_gbs": peak, "peak_kind": peak_kind,
@@ -521,6 +617,8 @@ def main():
                     help="diagnostic: identity page table instead of the workload's shuffled pages")
     ap.add_argument("--no-l2-flush", action="store_true",
                     help="do not write 256 MiB between timed steps (valid only where the step's own traffic exceeds L2)")
+    ap.add_argument("--flush-mode", default="write+read", choices=["write", "write+read"],
+                    help="how L2 is flushed between timed steps (see L2Flush)")
     ap.add_argument("--decode-loop", type=int, default=0,
                     help="also time this many consecutive decode steps (append, rebuild on block fill, step) and "
                          "report the amortised time per step")
@@ -529,12 +627,18 @@ def main():
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the other named configurations (the `other_workloads` list of the line)")
     ap.add_argument("--other-steps", type=int, default=20, help="timed steps per other configuration")
+    ap.add_argument("--phase-times", nargs="?", const="step", default=None, choices=["step", "score"],
+                    help="diagnostic, one GPU: run the timing build of the library and print where the time of one step "
+                         "(or of cobs_score_select alone) goes; not a benchmark value")
     ap.add_argument("--launch-selftest", action="store_true",
                     help="no GPU work: bring the N ranks up on gloo, run a stub step, print the line (tests the launch path)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    ensure_ranks(args)
-    if args.launch_selftest:
+    if not args.phase_times:
+        ensure_ranks(args)
+    if args.phase_times:
+        run_phase_times(args)
+    elif args.launch_selftest:
         run_launch_selftest(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -51,6 +51,15 @@ class Summaries(C.Structure):
 _lib = None
 
 
+def use_library(path: str):
+    """Load the library from `path` instead of the default build (before the first call): used by the benchmark's
+    phase-timing mode, which runs the build that carries the timing code."""
+    global _lib, LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("the library is already loaded")
+    LIB_PATH = path
+
+
 def lib():
     """Load libcobs.so once.  Raises if it has not been built (python -m paper_2607_09052_b200.build)."""
     global _lib

@@ -1,4 +1,7 @@
-"""Build the CUDA library in-tree: paper_2607_09052_b200/libcobs.so (sm_100a only)."""
+"""Build the CUDA library in-tree: paper_2607_09052_b200/libcobs.so (sm_100a only).
+
+`--timing` builds a second library, libcobs_timing.so, whose step kernel records per-warp phase timestamps
+(read by `bench.py --phase-times`); the production library carries no timing code."""
 
 from __future__ import annotations
 
@@ -10,6 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcobs.so")
+LIB_TIMING = os.path.join(HERE, "libcobs_timing.so")
 SOURCES = ["api.cu", "score_select.cu", "fused_step.cu", "summaries.cu", "exact_mass.cu", "adaptive.cu"]
 
 
@@ -18,31 +22,33 @@ def nvcc_path() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "cobs.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return LIB
+def build(force: bool = False, verbose: bool = False, timing: bool = False) -> str:
+    lib = LIB_TIMING if timing else LIB
+    if not force and not needs_build(lib):
+        return lib
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-    cmd += os.environ.get("COBS_NVCC_FLAGS", "").split()
+    if timing:
+        cmd += ["-DCOBS_TIMING"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
+    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", lib]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)
-        raise RuntimeError("nvcc failed building libcobs.so")
+        raise RuntimeError(f"nvcc failed building {os.path.basename(lib)}")
     if verbose:
         print(res.stdout + res.stderr)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, timing="--timing" in sys.argv))

@@ -2,6 +2,8 @@
 #include <cstdio>
 #include <cstring>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 #include <atomic>
@@ -83,11 +85,7 @@ static int choose_splits(const cobs_config *c) {
   // Two slices per streaming warp when the scoring runs in waves (then the second round of items absorbs the units
   // whose selection finishes last); one per warp otherwise (an item costs several microseconds beyond its bytes).
   const long long chunks = (long long)units * ((c->max_blocks + 15) / 16);
-#ifdef COBS_ITEMS_PER_WARP
-  const int per_warp = COBS_ITEMS_PER_WARP;
-#else
   const int per_warp = (chunks / kGridWarps >= 2) ? 2 : 1;
-#endif
   int s = per_warp * kGridWarps / units;
   const int need = (groups + kItemGroups - 1) / kItemGroups;
   if (s < need) s = need;

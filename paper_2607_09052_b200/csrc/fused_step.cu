@@ -65,18 +65,17 @@ constexpr int kFusedSmemBytes = kFWarps * kWarpSmemBytes;    // 225280: one CTA 
 constexpr long long kSpinLimit = 4000000;                    // x ~100 ns: bounded wait on another warp
 
 enum { PH_SCORE = 1, PH_ATTEND = 2 };
-#ifndef COBS_WAVES
-#define COBS_WAVES 4
-#endif
-constexpr int kWaves = COBS_WAVES;                           // the units are scored in this many waves
-#ifndef COBS_SCORE_RG
-#define COBS_SCORE_RG 4                                      // FP4 factor rows decoded and multiplied together
-#endif
+constexpr int kWaves = 4;                                    // the units are scored in this many waves
+constexpr int kScoreRowGroup = 4;                            // FP4 factor rows decoded and multiplied together
 
+// Phase timing (the build with -DCOBS_TIMING, `python -m paper_2607_09052_b200.build --timing`, which makes
+// libcobs_timing.so; read by `bench.py --phase-times`): every streaming warp records the global timer at its phase
+// boundaries and accumulates clock cycles per category inside the phases; the selection teams record when a unit
+// was complete and when its selection was published.  The production library carries none of this.
 #ifdef COBS_TIMING
-// development aid: per-warp phase boundary timestamps (ns), read back by cobs_debug_times
-__device__ unsigned long long g_dbg_times[4][4096];
-__device__ unsigned long long g_dbg_acc[8][4096];   // per-warp accumulated clock cycles by category
+__device__ unsigned long long g_dbg_times[4][4096];   // [start | scoring done | attention start | attention done][warp]
+__device__ unsigned long long g_dbg_acc[8][4096];     // accumulated clock cycles by category: attention [warp], scoring
+                                                      // [1200 + warp]; selection stamps (ns) [3000 + unit]
 __device__ __forceinline__ unsigned long long gtime() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -99,11 +98,19 @@ __device__ __forceinline__ unsigned long long gtime() {
 // ---------------------------------------------------------------------------------------------------
 // small PTX helpers
 // ---------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void cpa16(uint32_t dst, const void *src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src));
+// The summaries and the selected K / V are read exactly once per step: their copies carry an L2 evict-first policy,
+// so that they do not push the step's small shared state (block scores, chunk pairs, selections, split partials,
+// flags: written by one warp, read by another a few microseconds later) out of L2 and into the HBM queues.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
 }
-__device__ __forceinline__ void cpa16z(uint32_t dst, const void *src, int bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(bytes));
+__device__ __forceinline__ void cpa16(uint32_t dst, const void *src, uint64_t pol) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "l"(pol));
+}
+__device__ __forceinline__ void cpa16z(uint32_t dst, const void *src, int bytes, uint64_t pol) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;\n" ::"r"(dst), "l"(src), "r"(bytes), "l"(pol));
 }
 __device__ __forceinline__ void cpa4(uint32_t dst, const void *src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(dst), "l"(src));
@@ -115,6 +122,11 @@ __device__ __forceinline__ void cpa_wait() { asm volatile("cp.async.wait_group %
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ float lds_f32(uint32_t addr) {
@@ -178,6 +190,10 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
 }
 // Wait for the phase with the given parity to complete.  Bounded; false on expiry.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -465,6 +481,56 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid, int c
   }
 }
 
+// Curvature term of a 16-block chunk whose packed E2M1 rows are full width (128 codes: one 16-byte read per thread and
+// row) and whose rank R is a multiple of four: straight-line code, four rows (four independent accumulator chains) at
+// a time, the four scales of a block read in one go.  xa / xb: this thread's 16 bytes of row 0 of blocks 2 gid and
+// 2 gid + 1 (rows 64 bytes apart); sp: the scales of block 2 gid (those of block 2 gid + 1 follow them).
+// Adds sum_i (scale_i * (xi_i . q))^2 per block and head; the query's per-head factor is applied by the caller.
+template <int R, bool SCALE_F32>
+__device__ __forceinline__ void fp4_rows_full_width(uint32_t xa, uint32_t xb, uint32_t sp, const uint32_t (&bq)[8][2], float &sA0,
+                                                    float &sA1, float &sB0, float &sB1) {
+  static_assert(R % 4 == 0, "whole groups of four rows");
+#pragma unroll
+  for (int i0 = 0; i0 < R; i0 += 4) {
+    uint4 wa[4], wb[4];
+    float d[4][4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      wa[k] = lds128(xa + (i0 + k) * 64);
+      wb[k] = lds128(xb + (i0 + k) * 64);
+      d[k][0] = d[k][1] = d[k][2] = d[k][3] = 0.f;
+    }
+    float sa[4], sb[4];
+    if (SCALE_F32) {
+      const uint4 a = lds128(sp + i0 * 4), b = lds128(sp + R * 4 + i0 * 4);
+      sa[0] = __uint_as_float(a.x); sa[1] = __uint_as_float(a.y); sa[2] = __uint_as_float(a.z); sa[3] = __uint_as_float(a.w);
+      sb[0] = __uint_as_float(b.x); sb[1] = __uint_as_float(b.y); sb[2] = __uint_as_float(b.z); sb[3] = __uint_as_float(b.w);
+    } else {
+      const uint2 a = lds64(sp + i0 * 2), b = lds64(sp + R * 2 + i0 * 2);
+      const float2 a0 = __half22float2(*reinterpret_cast<const __half2 *>(&a.x)), a1 = __half22float2(*reinterpret_cast<const __half2 *>(&a.y));
+      const float2 b0 = __half22float2(*reinterpret_cast<const __half2 *>(&b.x)), b1 = __half22float2(*reinterpret_cast<const __half2 *>(&b.y));
+      sa[0] = a0.x; sa[1] = a0.y; sa[2] = a1.x; sa[3] = a1.y;
+      sb[0] = b0.x; sb[1] = b0.y; sb[2] = b1.x; sb[3] = b1.y;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint32_t ha[4], hb[4];
+        e2m1x8_to_f16(j == 0 ? wa[k].x : j == 1 ? wa[k].y : j == 2 ? wa[k].z : wa[k].w, ha);
+        e2m1x8_to_f16(j == 0 ? wb[k].x : j == 1 ? wb[k].y : j == 2 ? wb[k].z : wb[k].w, hb);
+        mma16816_f16(d[k][0], d[k][1], d[k][2], d[k][3], ha[0], hb[0], ha[1], hb[1], bq[2 * j][0], bq[2 * j][1]);
+        mma16816_f16(d[k][0], d[k][1], d[k][2], d[k][3], ha[2], hb[2], ha[3], hb[3], bq[2 * j + 1][0], bq[2 * j + 1][1]);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float d0 = d[k][0] * sa[k], d1 = d[k][1] * sa[k], d2 = d[k][2] * sb[k], d3 = d[k][3] * sb[k];
+      sA0 = fmaf(d0, d0, sA0); sA1 = fmaf(d1, d1, sA1); sB0 = fmaf(d2, d2, sB0); sB1 = fmaf(d3, d3, sB1);
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------
 // phase S: scoring (+ selection by the warp that completes a unit)
 // DT: COBS_SUMM_BF16 | COBS_SUMM_FP4_E2M1.  WPT: 32-bit words of codes per thread per FP4 row
@@ -520,8 +586,9 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     const int u0 = (units * w) / n_waves, u1 = (units * (w + 1)) / n_waves;
     const int tot = (u1 - u0) * cpu;                       // the host refuses configurations where this overflows
     // ceil-sized ranges: at the benchmark's size this leaves the last 20 CTAs without scoring work; they start on the
-    // attention of the first selected units while the others still score, which measured 5 us faster per step than
-    // equal shares for every warp
+    // attention of the first selected units while the others still score.  Equal shares for every warp end the
+    // scoring 5 us earlier and the step 4 us later (measured, several forms): the warps then reach the attention
+    // phase together, before most selections are published, and move through it in lockstep.
     const int per = (tot + n_wg - 1) / n_wg;
     cb = u0 * cpu + min(wg * per, tot);
     ce = u0 * cpu + min(wg * per + per, tot);
@@ -545,6 +612,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   };
 
   COBS_ACC_DECL;
+  const uint64_t pol = l2_evict_first_policy();
   // ---- bulk copies of (chunk c, batch b) into stage st; completion is counted on the stage's mbarrier ----
   // lanes 0-15 copy the factor rows of block `lane`, lanes 16-31 the mean of block `lane - 16`, lane 0 the scales
   auto issue = [&](int u, int ck, int n_sum, int b, int st) {
@@ -566,9 +634,9 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
       if (scales_bulk) tx += (uint32_t)(16 * r * scale_sz);
       mbar_expect_tx(bar, tx);
       if (single) {                            // the whole chunk: three contiguous pieces, one lane issues them
-        bulk_g2s(sbase, (const char *)p.mean + rec0 * (size_t)(D * 2), nblk * D * 2, bar);
-        if (rows > 0) bulk_g2s(sbase + xoff, (const char *)p.xi + rec0 * r * (size_t)ROWB, nblk * r * ROWB, bar);
-        if (scales_bulk) bulk_g2s(sbase + soff, (const char *)p.scale + rec0 * (size_t)(r * scale_sz), 16 * r * scale_sz, bar);
+        bulk_g2s(sbase, (const char *)p.mean + rec0 * (size_t)(D * 2), nblk * D * 2, bar, pol);
+        if (rows > 0) bulk_g2s(sbase + xoff, (const char *)p.xi + rec0 * r * (size_t)ROWB, nblk * r * ROWB, bar, pol);
+        if (scales_bulk) bulk_g2s(sbase + soff, (const char *)p.scale + rec0 * (size_t)(r * scale_sz), 16 * r * scale_sz, bar, pol);
       }
     }
     COBS_ACC(5);
@@ -583,14 +651,14 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
     __syncwarp();
     if (lane < 16) {
       if (lane < nblk && rows > 0)
-        bulk_g2s(sbase + xoff + lane * xs, (const char *)p.xi + ((rec0 + lane) * r + row0) * (size_t)ROWB, rows * ROWB, bar);
+        bulk_g2s(sbase + xoff + lane * xs, (const char *)p.xi + ((rec0 + lane) * r + row0) * (size_t)ROWB, rows * ROWB, bar, pol);
     } else if (b == 0 && lane - 16 < nblk) {
-      bulk_g2s(sbase + (lane - 16) * mrow, (const char *)p.mean + (rec0 + lane - 16) * (size_t)(D * 2), D * 2, bar);
+      bulk_g2s(sbase + (lane - 16) * mrow, (const char *)p.mean + (rec0 + lane - 16) * (size_t)(D * 2), D * 2, bar, pol);
     }
     if (FP4 && r > 0) {
       const char *ssrc = (const char *)p.scale + rec0 * (size_t)(r * scale_sz);
       if (scales_bulk) {
-        if (lane == 2) bulk_g2s(sbase + soff, ssrc, 16 * r * scale_sz, bar);
+        if (lane == 2) bulk_g2s(sbase + soff, ssrc, 16 * r * scale_sz, bar, pol);
       } else {                                // ragged last chunk of the array: plain loads, 4 bytes at a time
         for (int w = lane * 4; w < nblk * r * scale_sz; w += 128)
           *reinterpret_cast<uint32_t *>(wsm + st * kScoreStageBytes + soff + w) = *reinterpret_cast<const uint32_t *>(ssrc + w);
@@ -721,9 +789,25 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
       const int rows = min(r - row0, (cur_b == 0) ? ROWS0 : ROWSN);
       const uint32_t xs = (cur_b == 0) ? XS0 : XSN;
       const uint32_t xa = sbase + ((cur_b == 0) ? mean_bytes : 0) + (2 * gid) * xs + tig * (FP4 ? WPT * 4 : 16), xb = xa + xs;
-      if (FP4) {
+      bool rows_done = false;
+      if constexpr (FP4 && WPT == 4 && NT == 1) {
+        // the benchmark's descriptors (full key space, rank 4 or 8, the whole chunk in one stage): straight-line code
+        if (single && (r == 8 || r == 4)) {
+          const uint32_t spa = sbase + (kScoreStageBytes - scale_bytes) + (2 * gid) * r * scale_sz;
+          if (r == 8) {
+            if (scale_sz == 4) fp4_rows_full_width<8, true>(xa, xb, spa, bq[0], sA0, sA1, sB0, sB1);
+            else fp4_rows_full_width<8, false>(xa, xb, spa, bq[0], sA0, sA1, sB0, sB1);
+          } else {
+            if (scale_sz == 4) fp4_rows_full_width<4, true>(xa, xb, spa, bq[0], sA0, sA1, sB0, sB1);
+            else fp4_rows_full_width<4, false>(xa, xb, spa, bq[0], sA0, sA1, sB0, sB1);
+          }
+          rows_done = true;
+        }
+      }
+      if (rows_done) {
+      } else if (FP4) {
         // RG factor rows at a time: RG independent accumulator chains keep the tensor pipe busy
-        constexpr int RG = COBS_SCORE_RG;
+        constexpr int RG = kScoreRowGroup;
         const unsigned char *sp = wsm + st * kScoreStageBytes + (kScoreStageBytes - scale_bytes) + (2 * gid) * r * scale_sz;
 #pragma unroll 1
         for (int i0 = 0; i0 < ROWS_MAX; i0 += RG) {
@@ -903,6 +987,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
 
   // items are handed out in unit order from a global counter: a warp that arrives late simply takes fewer
   const int n_items = units * n_splits;
+  const uint64_t pol = l2_evict_first_policy();
   COBS_ACC_DECL;
 
   // Closing an item = making its partial visible, counting it, and merging the unit if it was the last slice.
@@ -1084,13 +1169,13 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
           const int nv = T - first;
           if (nv >= 16) {
 #pragma unroll
-            for (int j = 0; j < NCP; ++j) { cpa16(dst + cdst[j], ks + 32 * j); cpa16(dst + VOFF + cdst[j], vs + 32 * j); }
+            for (int j = 0; j < NCP; ++j) { cpa16(dst + cdst[j], ks + 32 * j, pol); cpa16(dst + VOFF + cdst[j], vs + 32 * j, pol); }
           } else {                             // ragged tail: rows past the end of the sequence are zero filled
 #pragma unroll
             for (int j = 0; j < NCP; ++j) {
               const int bytes = ((lane + 32 * j) / CH < nv) ? 16 : 0;
-              cpa16z(dst + cdst[j], ks + 32 * j, bytes);
-              cpa16z(dst + VOFF + cdst[j], vs + 32 * j, bytes);
+              cpa16z(dst + cdst[j], ks + 32 * j, bytes, pol);
+              cpa16z(dst + VOFF + cdst[j], vs + 32 * j, bytes, pol);
             }
           }
         }
@@ -1608,9 +1693,9 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
   const int *seq_lens = p.seq_lens;
   if (p.B <= kLenCache) {
     for (int i = threadIdx.x; i < p.B; i += kFThreads) s_len[i] = p.seq_lens[i];
-    __syncthreads();
     seq_lens = s_len;
   }
+  __syncthreads();
   if (warp < kFWarps) {
     // ---- streaming warps: score their chunks, then attend their items -------------------------------------
     unsigned char *wsm = fsm + warp * kWarpSmemBytes;

@@ -32,7 +32,7 @@ def run_stage_s(wl, inp_cpu=None, units=None, inp_dev=None, summ=None):
     if inp_dev is None:
         inp_cpu = synth.generate(wl) if inp_cpu is None else inp_cpu
         inp_dev = to_dev(inp_cpu)
-    src = inp_dev if inp_cpu is None else inp_cpu
+    src = inp_dev if inp_cpu is None else inp_cpu      # where the oracle reads its inputs from
     cfg = B.make_config(wl)
     kv = B.make_kv(inp_dev)
     if summ is None:
@@ -145,7 +145,74 @@ def test_cfg4_full_size_sampled_units():
     ws = B.alloc_workspace(cfg, "cuda")
     B.cobs_build_summaries(cfg, B.make_kv(inp), 0, wl.max_blocks, summ, ws)
     assert B.cobs_read_status(ws) == 0
-    run_stage_s(wl, inp_dev=inp, units=[(0, 0), (7, 3), (15, 7)], summ=summ)
+    # the 128 units are scored in four waves of 32: the first and the last unit of every wave, and one inside
+    units = [(0, 0), (3, 7), (4, 0), (7, 3), (7, 7), (8, 0), (11, 7), (12, 0), (15, 7)]
+    run_stage_s(wl, inp_dev=inp, units=units, summ=summ)
+    check_fused_equals_two_calls_on_every_unit(wl, inp, summ)
+
+
+def check_fused_equals_two_calls_on_every_unit(wl, inp, summ):
+    """For EVERY unit (no oracle time needed): cobs_decode_step selects exactly what cobs_score_select selects, and
+    its output is cobs_sparse_decode's on that selection up to fp32 reassociation."""
+    B = _binding()
+    cfg = B.make_config(wl)
+    kv = B.make_kv(inp)
+    ws = B.alloc_workspace(cfg, "cuda")
+    nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+    sel = torch.full((nb, hkv, wl.topk), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((nb, hkv), -7, dtype=torch.int32, device="cuda")
+    B.cobs_score_select(cfg, inp["q"], summ, inp["seq_lens"], sel, cnt, None, ws)
+    out_a = torch.zeros((nb, hq, D), dtype=torch.float32, device="cuda")
+    lse_a = torch.zeros((nb, hq), dtype=torch.float32, device="cuda")
+    B.cobs_sparse_decode(cfg, inp["q"], kv, sel, cnt, out_a, lse_a, ws)
+    sel_f, cnt_f = torch.full_like(sel, -7), torch.full_like(cnt, -7)
+    out_f, lse_f = torch.zeros_like(out_a), torch.zeros_like(lse_a)
+    B.cobs_decode_step(cfg, inp["q"], kv, summ, out_f, lse_f, sel_f, cnt_f, ws)
+    assert B.cobs_read_status(ws) == 0
+    assert torch.equal(sel, sel_f) and torch.equal(cnt, cnt_f)
+    lens = inp["seq_lens"].cpu().tolist()
+    want = torch.tensor([min(wl.topk, O.window_start(t, wl.window, wl.block_size) // wl.block_size) for t in lens],
+                        dtype=torch.int32)
+    assert torch.equal(cnt.cpu(), want[:, None].expand(nb, hkv))
+    s = sel.cpu()
+    for b in range(nb):                                       # ascending, distinct, candidates only, -1 padding
+        k = int(want[b])
+        assert torch.all(s[b, :, k:] == -1)
+        if k:
+            assert torch.all(s[b, :, :k] >= 0) and torch.all(s[b, :, :k] < O.window_start(lens[b], wl.window, wl.block_size) // wl.block_size)
+            assert torch.all(s[b, :, 1:k] > s[b, :, :k - 1])
+    scale = out_a.abs().amax(dim=-1, keepdim=True).clamp_min(1e-30)
+    assert float(((out_f - out_a).abs() / scale).max()) <= 1e-5
+    assert float((lse_f - lse_a).abs().max()) <= 1e-5
+
+
+def test_cfg5_full_size_sampled_units():
+    """Configuration 5 at full size (8 sequences x 64k, blocks of 128, groups of 8 heads), as the benchmark runs it."""
+    B = _binding()
+    wl = WL["cfg5_64k_g8"]
+    inp = synth.generate(wl, "cuda")
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    B.cobs_build_summaries(cfg, B.make_kv(inp), 0, wl.max_blocks, summ, ws)
+    assert B.cobs_read_status(ws) == 0
+    run_stage_s(wl, inp_dev=inp, units=[(0, 0), (3, 5), (7, 7)], summ=summ)
+    check_fused_equals_two_calls_on_every_unit(wl, inp, summ)
+
+
+def test_cfg3a_full_batch_sampled_units():
+    """Configuration 3A (subspace descriptor, packed E2M1) at its full batch of four sequences."""
+    B = _binding()
+    wl = WL["cfg3a_32k_subspace"]
+    cpu = synth.generate(wl)
+    inp = to_dev(cpu)
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda", inp.get("u_q"))
+    ws = B.alloc_workspace(cfg, "cuda")
+    B.cobs_build_summaries(cfg, B.make_kv(inp), 0, wl.max_blocks, summ, ws)
+    assert B.cobs_read_status(ws) == 0
+    run_stage_s(wl, inp_cpu=cpu, inp_dev=inp, units=[(0, 0), (1, 6), (2, 3), (3, 7)], summ=summ)
+    check_fused_equals_two_calls_on_every_unit(wl, inp, summ)
 
 
 # --- the opt-in tcgen05 scoring path ------------------------------------------------------------------------
@@ -544,6 +611,130 @@ def test_quantiser_bit_exact(scale_dtype, ds):
     assert np.array_equal(scale.float().cpu().numpy(), scale_ref)
 
 
+def test_e2m1_rounding_rule_agrees_with_the_hardware_conversion():
+    """The oracle's E2M1 rounding (nearest, ties to the even mantissa bit, saturating at 6) against the GPU's own
+    conversion instruction on a dense fp32 grid over [-6, 6], every tie point with both fp32 neighbours, and
+    values beyond the range.  Every row holds a 6, so the oracle's scale is exactly 1 and t = x."""
+    B = _binding()
+    ties = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], np.float32)
+    near = np.concatenate([ties, np.nextafter(ties, np.float32(0)), np.nextafter(ties, np.float32(10))])
+    special = np.concatenate([near, -near, np.array([0.0, 0.5, 1, 1.5, 2, 3, 4, 6, -0.5, -1, -1.5, -2, -3, -4, -6,
+                                                      1e-30, 1e-45, 0.2499999, 5.9999995], np.float32)])
+    dense = np.linspace(-6.0, 6.0, 400001).astype(np.float32)
+    rnd = (np.random.default_rng(0).uniform(-6, 6, 200000)).astype(np.float32)
+    vals = np.concatenate([special, dense, rnd])
+    cols = 127
+    vals = np.concatenate([vals, np.zeros((-len(vals)) % cols, np.float32)]).reshape(-1, cols)
+    rows = np.concatenate([np.full((vals.shape[0], 1), 6.0, np.float32), vals], axis=1)     # max |x| = 6 -> scale 1
+    codes_ref, scale_ref = O.quantise_e2m1(rows, "fp32")
+    assert np.all(scale_ref == 1.0)
+    x = torch.from_numpy(rows.reshape(-1)).cuda()
+    hw = torch.zeros(x.numel(), dtype=torch.uint8, device="cuda")
+    B.cobs_hw_e2m1_codes(x, hw)
+    hw = hw.cpu().numpy().reshape(rows.shape)
+    assert np.array_equal(hw & 7, codes_ref & 7)                  # the magnitude index, everywhere
+    nz = (codes_ref & 7) != 0
+    assert np.array_equal(hw[nz] >> 3, codes_ref[nz] >> 3)        # the sign wherever the value is not zero
+    # beyond the largest magnitude the conversion saturates, as the oracle's last threshold does (t > 5 -> 6)
+    big = torch.tensor([6.5, 7.0, 100.0, 3e38, -6.5, -7.0, -1e9], dtype=torch.float32, device="cuda")
+    hb = torch.zeros(big.numel(), dtype=torch.uint8, device="cuda")
+    B.cobs_hw_e2m1_codes(big, hb)
+    assert hb.cpu().tolist() == [7, 7, 7, 7, 15, 15, 15]
+    # codes that are zero in magnitude: +0 and tiny positives give code 0 on both sides.  Negative values that
+    # round to zero keep their sign bit in the oracle's rule (code 8, which decodes to the same 0)
+    zero_neg = torch.tensor([-0.0, -1e-30, -0.2], dtype=torch.float32, device="cuda")
+    hz = torch.zeros(3, dtype=torch.uint8, device="cuda")
+    B.cobs_hw_e2m1_codes(zero_neg, hz)
+    assert all(int(c) & 7 == 0 for c in hz.cpu().tolist())
+
+
+@pytest.mark.parametrize("topk", [16, 64])
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+def test_selection_with_few_heavy_blocks_over_a_flat_background(G, topk):
+    """Units of 513 ... 1024 summarised blocks whose scores are a handful of heavy blocks over a nearly uniform
+    background: at some bisection round of the top-k more than 512 keys lie above the lowest trial value while
+    fewer than k lie above the others (the case in which a packed count once overflowed its field).  Selection
+    against the oracle, and nothing may be written outside a unit's own row of sel_idx (guard rows)."""
+    B = _binding()
+    L, D, NB = 16, 64, 1024
+    n_sums = [600, 1023, 1024, 513, 512, 700]
+    lens = [n * L + (3 if n < NB else 0) for n in n_sums]
+    wl = synth.Workload("flat", len(lens), G, 1, D, NB * L, L, 16, rank=2, topk=topk, window=L + 5, summary_dtype="bf16",
+                        key_model="iid", seed=31 + G, seq_lens=lens)
+    inp = synth.generate(wl)
+    gen = torch.Generator().manual_seed(100 + G)
+    v = torch.randn(D, generator=gen)
+    inp["q"] = (v[None, None, :] + 0.2 * torch.randn(len(lens), G, D, generator=gen)).to(torch.bfloat16)
+    dev = to_dev(inp)
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    mean_v, xi_v, _ = B.summary_views(cfg, summ)
+    # background: means -0.3 v plus a little noise (scores within a few per cent of each other); 4 heavy blocks
+    mean_all = (-0.3 * v[None, None, :] + 0.004 * torch.randn(len(lens), NB, D, generator=gen))
+    heavy = [[int(x) for x in torch.randperm(n - 4, generator=gen)[:4]] for n in n_sums]
+    for i, hb in enumerate(heavy):
+        mean_all[i, hb] = 0.6 * v
+    mean_bf = mean_all.to(torch.bfloat16)
+    xi_bf = (0.05 * torch.randn(len(lens), NB, 2, D, generator=gen)).to(torch.bfloat16)
+    mean_v[:, 0] = mean_bf.cuda()
+    xi_v[:, 0] = xi_bf.cuda()
+    guard = torch.full((len(lens) + 2, topk), -7, dtype=torch.int32, device="cuda")
+    sel = guard[1:-1].view(len(lens), 1, topk)
+    cnt = torch.full((len(lens), 1), -7, dtype=torch.int32, device="cuda")
+    B.cobs_score_select(cfg, dev["q"], summ, dev["seq_lens"], sel, cnt, None, ws)
+    guard_f = torch.full_like(guard, -7)
+    sel_f = guard_f[1:-1].view(len(lens), 1, topk)
+    cnt_f = torch.full_like(cnt, -7)
+    out = torch.zeros((len(lens), G, D), dtype=torch.float32, device="cuda")
+    B.cobs_decode_step(cfg, dev["q"], B.make_kv(dev), summ, out, None, sel_f, cnt_f, ws)
+    assert B.cobs_read_status(ws) == 0
+    for g_ in (guard, guard_f):
+        assert torch.all(g_[0] == -7) and torch.all(g_[-1] == -7)
+    sel_c, sel_fc = sel.cpu(), sel_f.cpu()
+    for i, n_sum in enumerate(n_sums):
+        n_cand = O.window_start(lens[i], wl.window, L) // L
+        e = O.log_mass_estimates(inp["q"][i].double().numpy(), mean_bf[i, :n_sum].double().numpy(),
+                                 xi_bf[i, :n_sum].double().numpy(), L)
+        score = O.group_scores(e)
+        ref = set(int(x) for x in O.select_topk(score, n_cand, topk))
+        assert set(heavy[i]) <= ref                               # the heavy blocks are the top of the list
+        for which, got in (("cobs_score_select", sel_c[i, 0]), ("cobs_decode_step", sel_fc[i, 0])):
+            ok, msg, _ = check_selection(got.tolist(), score, n_cand, topk)
+            assert ok, (which, n_sum, msg)
+
+
+def test_length_beyond_the_page_table_is_reported_not_followed():
+    """T = NB * L + L - 1 with a page table that covers exactly NB * L tokens: the window's last tokens have no
+    page-table entry.  The kernel must not read past the row: it skips them and leaves COBS_ERR_BOUNDS."""
+    B = _binding()
+    wl = WL["cfg1_tiny"].replace(summary_dtype="bf16")
+    assert wl.max_pages_per_seq * wl.page_size == wl.max_blocks * wl.block_size
+    cpu = synth.generate(wl)
+    inp = to_dev(cpu)
+    cfg = B.make_config(wl)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    kv = B.make_kv(inp)
+    B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, summ, ws)
+    # the page table is the last thing in its allocation's row: put a poisoned row behind it
+    table = torch.full((wl.batch + 1, wl.max_pages_per_seq), 2 ** 30, dtype=torch.int32, device="cuda")
+    table[:wl.batch] = inp["page_table"]
+    inp["page_table"] = table[:wl.batch]
+    kv = B.make_kv(inp)
+    inp["seq_lens"].fill_(wl.max_blocks * wl.block_size + wl.block_size - 1)
+    out = torch.zeros((wl.batch, wl.n_q_heads, wl.head_dim), dtype=torch.float32, device="cuda")
+    B.cobs_decode_step(cfg, inp["q"], kv, summ, out, None, None, None, ws)
+    assert B.cobs_read_status(ws) == 6
+    B.cobs_reset_status(ws)
+    # the tokens that do have a page were served: same result as the full-capacity length, whose window is those tokens
+    assert torch.isfinite(out).all()
+    inp["seq_lens"].fill_(wl.max_blocks * wl.block_size)
+    out2 = torch.zeros_like(out)
+    B.cobs_decode_step(cfg, inp["q"], kv, summ, out2, None, None, None, ws)
+    assert B.cobs_read_status(ws) == 0
+
+
 # --- builder (backward error; eigenvectors of close eigenvalues are not unique to rounding) ---------------------
 
 def check_builder(wl, units):
@@ -615,7 +806,14 @@ def check_builder(wl, units):
             scale = torch.zeros(flat.shape[0], dtype=scale_s.dtype, device="cuda")
             B.cobs_quantise_xi(cfg, flat, codes, scale)
             assert torch.equal(codes.view_as(xi_s), xi_s) and torch.equal(scale.view_as(scale_s), scale_s)
-            # and against the oracle's quantiser applied to the oracle's own factors: informational agreement
+            # and the ORACLE's quantiser applied to the device's fp32 factors gives the device's codes and scales,
+            # bit for bit (the builder's own FP4 output against the paper-side definition of the format)
+            codes_ref, scale_ref = O.quantise_e2m1(flat.cpu().numpy(), wl.scale_dtype)
+            ds_pad = B.cobs_padded_sub_dim(cfg)
+            got = B.unpack_fp4_rows(xi_s.reshape(-1, ds_pad // 2), ds_pad).cpu().numpy()
+            assert np.array_equal(got[:, :ds], codes_ref)
+            assert np.all(got[:, ds:] == 0)
+            assert np.array_equal(scale_s.reshape(-1).float().cpu().numpy(), scale_ref)
     assert B.cobs_read_status(ws) == 0
 
 

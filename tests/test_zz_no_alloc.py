@@ -7,17 +7,20 @@ import pytest
 import torch
 
 from paper_2607_09052_b200 import synth
-from parity import OUT_TOL, out_rel_err
+from parity import OUT_TOL, oracle_attend, out_rel_err
 
 pytestmark = pytest.mark.gpu
 
 
 def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row():
     from paper_2607_09052_b200 import binding as B
-    wl = synth.named_workloads()["cfg4_128k"].replace(batch=3, seq_len=8192)
-    cfg = B.make_config(wl)
-    ws = B.alloc_workspace(cfg, "cuda")
-    for call, seed in enumerate((41, 42)):
+    base = synth.named_workloads()["cfg4_128k"]
+    # the second call has another batch, context and top-k: it finds the first call's counters and partials laid
+    # out differently in the shared scratch
+    for call, (seed, batch, seq_len, topk) in enumerate(((41, 3, 8192, 64), (42, 2, 4096, 24))):
+        wl = base.replace(batch=batch, seq_len=seq_len, topk=topk)
+        cfg = B.make_config(wl)
+        ws = B.alloc_workspace(cfg, "cuda")
         cpu = synth.generate(wl.replace(seed=seed))
         inp = {k: (v.cuda() if k != "planted" else v) for k, v in cpu.items()}
         kv = B.make_kv(inp)
@@ -39,6 +42,14 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
         err = out_rel_err(out_st.cpu().numpy(), out_ws.cpu().double().numpy())
         assert np.all(err <= OUT_TOL), (call, err.max())
         assert np.allclose(lse_st.cpu().numpy(), lse_ws.cpu().numpy(), atol=2e-3, rtol=0), call
+        # and against the CPU oracle's attention over the same blocks, on two units
+        G = wl.group
+        for (b, h) in ((0, 0), (batch - 1, wl.n_kv_heads - 1)):
+            chosen = [int(x) for x in sel[b, h].cpu() if x >= 0]
+            ref_out, ref_lse = oracle_attend(wl, cpu, b, h, chosen)
+            hs = slice(h * G, (h + 1) * G)
+            assert np.all(out_rel_err(out_st[b, hs].cpu().numpy(), ref_out) <= OUT_TOL), (call, b, h)
+            assert np.allclose(lse_st[b, hs].cpu().numpy(), ref_lse, atol=2e-3, rtol=0), (call, b, h)
 
 
 def test_static_scratch_variant_refuses_what_does_not_fit():
