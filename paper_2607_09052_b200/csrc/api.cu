@@ -138,6 +138,7 @@ static void fill_params(Params &p, const cobs_config *c, void *workspace) {
     p.status = reinterpret_cast<int32_t *>(base + w.status);
     p.ctl_done = reinterpret_cast<int *>(base + w.status) + 1;
     p.ctl_item = reinterpret_cast<int *>(base + w.status) + 2;
+    p.ctl_bar = reinterpret_cast<int *>(base + w.status) + 3;
     p.ctl_score = reinterpret_cast<int *>(base + w.ctl);
     p.ctl_ready = p.ctl_score + (size_t)p.B * p.Hkv;
     p.ctl_att = p.ctl_ready + (size_t)p.B * p.Hkv;

@@ -35,11 +35,12 @@ struct Params {
   int32_t *status;
   int *ctl_done;              // CTAs of the persistent kernel that have finished
   int *ctl_item;              // next attention item to hand out
+  int *ctl_bar;               // CTAs that have passed the grid barrier after the query projection
   int *ctl_score;             // [B * Hkv] scored chunks per unit
   int *ctl_ready;             // [B * Hkv] 1 once the unit's selection is written
   int *ctl_att;               // [B * Hkv] attention slices finished per unit
-  const float *qtilde;        // [B][Hq][Ds_pad] prepared subspace query, or NULL
-  float *qtilde_out;
+  const float *qtilde;        // [B][Hq][Ds_pad] projected subspace query (what the scoring reads), or NULL
+  float *qtilde_out;          // where the step kernel's prologue writes it (workspace)
   float *e;                   // [B][Hkv][G][NB]
   float *lse_part;            // [B][Hkv][G][ceil(NB / 16)][2] per-chunk (max, sum-exp) of e
   float *partial;             // [B][Hkv][n_splits] slices of [G][D] accumulators + [G] (max, sum) pairs

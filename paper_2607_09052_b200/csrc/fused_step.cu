@@ -482,7 +482,7 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid, int c
 }
 
 // Curvature term of a 16-block chunk whose packed E2M1 rows are full width (128 codes: one 16-byte read per thread and
-// row) and whose rank R is a multiple of four: straight-line code, four rows (four independent accumulator chains) at
+// row) and whose rank R is a multiple of four: no clamps or row tests, four rows (four independent accumulator chains) at
 // a time, the four scales of a block read in one go.  xa / xb: this thread's 16 bytes of row 0 of blocks 2 gid and
 // 2 gid + 1 (rows 64 bytes apart); sp: the scales of block 2 gid (those of block 2 gid + 1 follow them).
 // Adds sum_i (scale_i * (xi_i . q))^2 per block and head; the query's per-head factor is applied by the caller.
@@ -490,7 +490,7 @@ template <int R, bool SCALE_F32>
 __device__ __forceinline__ void fp4_rows_full_width(uint32_t xa, uint32_t xb, uint32_t sp, const uint32_t (&bq)[8][2], float &sA0,
                                                     float &sA1, float &sB0, float &sB1) {
   static_assert(R % 4 == 0, "whole groups of four rows");
-#pragma unroll
+#pragma unroll 1                                 // rolled: half the code at rank 8 (instruction fetch is a visible stall of this kernel)
   for (int i0 = 0; i0 < R; i0 += 4) {
     uint4 wa[4], wb[4];
     float d[4][4];
@@ -733,7 +733,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
                 const float4 *src = reinterpret_cast<const float4 *>(
                     p.qtilde + ((size_t)b_idx * p.Hq + h * G + gid) * p.Ds_pad + tig * (WPT * 8) + j * 8);
                 float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-                if (gid < G) { lo = src[0]; hi = src[1]; }
+                if (gid < G) { lo = __ldcg(src); hi = __ldcg(src + 1); }
                 e[j][0] = lo.x; e[j][1] = lo.y; e[j][2] = lo.z; e[j][3] = lo.w;
                 e[j][4] = hi.x; e[j][5] = hi.y; e[j][6] = hi.z; e[j][7] = hi.w;
               } else {
@@ -1680,6 +1680,67 @@ __device__ void umma_epilogue(const Params &p, const UmmaList &l, unsigned char 
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Prologue of the subspace descriptor: q~ = U_Q^T (q / sqrt(D)) for every query head, zero padded to Ds_pad - the
+// one O(s D) projection per step and head that the scoring then shares across all blocks (Method, "Per-step
+// scoring").  Teams of four warps take (head, 32 consecutive subspace coordinates) tasks: lane = coordinate, so the
+// reads of U_Q [Hkv][D][Ds] are coalesced; each warp sums a quarter of the head dimension (all its loads in flight at
+// once) and the quarters are added in a fixed order.  The result goes to the workspace; a grid barrier (the launch
+// is cooperative, so every CTA is resident) makes it visible before any warp scores.
+// ---------------------------------------------------------------------------------------------------
+__device__ void project_queries(const Params &p) {
+  __shared__ float s_part[16][32];                // partial sums of the CTA's warps (at most 16 warps)
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int teams = (int)(blockDim.x >> 5) / 4;   // four warps share a task: each sums a quarter of the head dimension
+  const int team = warp >> 2, quarter = warp & 3;
+  const int nsb = p.Ds_pad / 32, n_tasks = p.B * p.Hq * nsb;
+  const int dq = p.D / 4;                         // 32 or 16 coordinates per quarter: all their loads fly together
+  const float inv_sqrt_d = 1.0f / sqrtf((float)p.D);
+  for (int base = blockIdx.x * teams; base < n_tasks; base += gridDim.x * teams) {
+    const int t = base + team;
+    const bool active = team < teams && t < n_tasks;
+    float v = 0.f;
+    int bh = 0, sidx = 0;
+    if (active) {
+      bh = t / nsb;
+      const int sb = t - bh * nsb, hq = bh % p.Hq, h = hq / p.G;
+      sidx = sb * 32 + lane;
+      const float qv = (lane < dq) ? __bfloat162float(p.q[(size_t)bh * p.D + quarter * dq + lane]) * inv_sqrt_d : 0.f;
+      const bool live = sidx < p.Ds;              // padding coordinates take part in the shuffles and end as 0
+      const float *uq = p.u_q + ((size_t)h * p.D + quarter * dq) * p.Ds + (live ? sidx : 0);
+      float x[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) x[j] = (live && j < dq) ? __ldg(uq + (size_t)j * p.Ds) : 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v = fmaf(x[j], __shfl_sync(0xffffffffu, qv, j), v);
+    }
+    if (warp < 16) s_part[warp][lane] = v;
+    __syncthreads();
+    if (active && quarter == 0)                   // fixed order: the same bits every time
+      __stcg(p.qtilde_out + (size_t)bh * p.Ds_pad + sidx,
+             ((s_part[warp][lane] + s_part[warp + 1][lane]) + s_part[warp + 2][lane]) + s_part[warp + 3][lane]);
+    __syncthreads();
+  }
+}
+
+// Every CTA of the (cooperatively launched, hence fully resident) grid has arrived and its writes are visible.
+// Bounded: on expiry COBS_ERR_TIMEOUT is recorded and the caller goes on (its results are then undefined).
+__device__ void grid_barrier(const Params &p) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(p.ctl_bar, 1);
+    bool ok = false;
+    for (long long it = 0; it < kSpinLimit; ++it) {
+      if (ld_volatile(p.ctl_bar) >= (int)gridDim.x) { ok = true; break; }
+      __nanosleep(50);
+    }
+    if (!ok) report(p.status, COBS_ERR_TIMEOUT);
+    __threadfence();
+  }
+  __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------------
 template <int DT, int D, int WPT, int NT>
@@ -1696,6 +1757,10 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
     seq_lens = s_len;
   }
   __syncthreads();
+  if ((phases & PH_SCORE) && p.u_q) {
+    project_queries(p);
+    grid_barrier(p);
+  }
   if (warp < kFWarps) {
     // ---- streaming warps: score their chunks, then attend their items -------------------------------------
     unsigned char *wsm = fsm + warp * kWarpSmemBytes;
@@ -1726,7 +1791,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
   if (is_last) {
     const int units = p.B * p.Hkv;
     for (int i = threadIdx.x; i < units; i += kFThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
-    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; }
+    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; *p.ctl_bar = 0; }
   }
 }
 
@@ -1798,31 +1863,7 @@ __global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p,
   if (is_last) {
     const int units = p.B * p.Hkv;
     for (int i = threadIdx.x; i < units; i += kUThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
-    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; }
-  }
-}
-
-// q~ = U_Q^T (q / sqrt(D)) for every query head, zero padded to Ds_pad (subspace descriptor only).
-__global__ void qtilde_kernel(Params p) {
-  const int bh = blockIdx.x, b_idx = bh / p.Hq, hq = bh - b_idx * p.Hq, h = hq / p.G;
-  extern __shared__ float qs[];
-  const float inv_sqrt_d = 1.0f / sqrtf((float)p.D);
-  for (int d = threadIdx.x; d < p.D; d += blockDim.x) qs[d] = __bfloat162float(p.q[(size_t)bh * p.D + d]) * inv_sqrt_d;
-  __syncthreads();
-  for (int s = threadIdx.x; s < p.Ds_pad; s += blockDim.x) {
-    float v = 0.f;
-    if (s < p.Ds) {
-      const float *uq = p.u_q + (size_t)h * p.D * p.Ds + s;
-      // 16 loads in flight at a time (the products are summed in the same order as a plain loop)
-      for (int d0 = 0; d0 < p.D; d0 += 16) {
-        float x[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) x[j] = __ldg(uq + (size_t)(d0 + j) * p.Ds);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) v = fmaf(x[j], qs[d0 + j], v);
-      }
-    }
-    p.qtilde_out[(size_t)bh * p.Ds_pad + s] = v;
+    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; *p.ctl_bar = 0; }
   }
 }
 
@@ -1941,13 +1982,6 @@ static cudaError_t launch_fused_umma(Params p, int phases, cudaStream_t stream) 
 }
 
 cudaError_t launch_fused(const Params &p, int phases, cudaStream_t stream) {
-  if ((phases & PH_SCORE) && p.u_q) {
-    Params q = p;
-    qtilde_kernel<<<p.B * p.Hq, 128, p.D * sizeof(float), stream>>>(q);
-    count_launch();
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-  }
   if ((phases & PH_SCORE) && umma_score_supported(p)) {
     const cudaError_t e = launch_fused_umma(p, phases, stream);
     if (e != cudaErrorNotSupported) return e;                // not supported: too many units per CTA, or no encoder
@@ -2017,6 +2051,7 @@ extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void 
   p.status = reinterpret_cast<int32_t *>(base);
   p.ctl_done = reinterpret_cast<int *>(base) + 1;
   p.ctl_item = reinterpret_cast<int *>(base) + 2;
+  p.ctl_bar = reinterpret_cast<int *>(base) + 3;
   p.ctl_score = reinterpret_cast<int *>(base + kStatusBytes);
   p.ctl_ready = p.ctl_score + units;
   p.ctl_att = p.ctl_ready + units;
