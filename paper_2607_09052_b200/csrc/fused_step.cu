@@ -234,7 +234,7 @@ __device__ __forceinline__ void team_sync() { asm volatile("bar.sync 1, %0;\n" :
 // use: one round trip.  Needs NB % 4 == 0.
 // PPC: (max, sum) pairs per 16-block chunk and head left by the scoring path (1, or 4 = one per four blocks).
 template <int PPC, int BPT>
-__device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int tid) {
+__device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int tid, int part) {
   static_assert(BPT == 4 || BPT == 8 || BPT == 16, "blocks per thread");
   static_assert(kSelWarps == 4, "one 16-byte read takes the four warps' words");
   constexpr int NQ = BPT / 4;                    // groups of four blocks of a thread
@@ -253,6 +253,13 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
   float2 pr[8];                                  // (max, sum) of chunk `tid`, per head (threads below n_chunks)
   float own_m[8][NQ];                            // max of the chunk part each of this thread's groups lies in
   float4 x[GB][NQ];
+  float sc[BPT];
+  uint32_t keys[BPT];
+#pragma unroll
+  for (int j = 0; j < BPT; ++j) { sc[j] = 0.f; keys[j] = 0u; }
+  // part < 0: the selection proper.  part = 0 .. 3: a rehearsal of one quarter of this code by one warp alone (no
+  // barrier, nothing written), see select_team.
+  const bool real = part < 0, dry = !real;
   auto load_t = [&](int g0) {
 #pragma unroll
     for (int g = 0; g < GB; ++g)
@@ -266,6 +273,14 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
     pr[g] = make_float2(-INFINITY, 0.f);
 #pragma unroll
     for (int q = 0; q < NQ; ++q) own_m[g][q] = -INFINITY;
+  }
+#pragma unroll
+  for (int g = 0; g < GB; ++g)
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) x[g][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (real || part == 0) {
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
     if (g < G) {
       if (PPC == 1) {
         if (loader) pr[g] = __ldcg(pp + (size_t)g * cpu + tid);
@@ -317,12 +332,11 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
       if (lane == 0) { s_m[g][warp] = M; s_s[g][warp] = sum; }
     }
   }
+  }
   COBS_SEL_STAMP(2);
-  team_sync();
+  if (real) team_sync();
   // ---- scores of this thread's blocks: score_b = sum_g t[g][b] * exp(part max[g] - lse_g) -----------------------
-  float sc[BPT];
-#pragma unroll
-  for (int j = 0; j < BPT; ++j) sc[j] = 0.f;
+  if (real || part == 1) {
 #pragma unroll
   for (int g0 = 0; g0 < 8; g0 += GB) {
     if (g0 < G) {
@@ -348,24 +362,28 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
       }
     }
   }
-  uint32_t keys[BPT];
 #pragma unroll
   for (int j = 0; j < BPT; ++j) {
     const int b = b0 + j;
     if (b >= n_sum) sc[j] = 0.f;                 // beyond the summarised blocks nothing was written
-    if (p.scores && b < n_sum) p.scores[(size_t)u * NB + b] = sc[j];
+    if (p.scores && b < n_sum && !dry) p.scores[(size_t)u * NB + b] = sc[j];
     keys[j] = (b < n_cand) ? __float_as_uint(sc[j]) : 0u;
+  }
   }
   COBS_SEL_STAMP(3);
   // ---- top-k ------------------------------------------------------------------------------------------------
   int32_t *out = p.sel_idx + (size_t)u * p.topk;
   const int k = min(p.topk, n_cand);
-  if (tid == 0) p.sel_cnt[u] = k;
-  for (int i = k + tid; i < p.topk; i += kSelThreads) out[i] = -1;
-  if (k == n_cand) {
-    for (int i = tid; i < k; i += kSelThreads) out[i] = i;
-    return;
+  uint32_t theta = 0u;
+  if (real) {
+    if (tid == 0) p.sel_cnt[u] = k;
+    for (int i = k + tid; i < p.topk; i += kSelThreads) out[i] = -1;
+    if (k == n_cand) {
+      for (int i = tid; i < k; i += kSelThreads) out[i] = i;
+      return;
+    }
   }
+  if (real || part == 2) {
   // k-th largest key by bisection on its bits (scores are >= 0, so their bit patterns order like integers):
   // theta = the largest T with #(key >= T) >= k.  Bit 30 alone, then two bits per round: three trial values, whose
   // counts travel packed as unsigned fields (11, 11 and 10 bits of one word while a team holds at most 512 keys - no
@@ -378,7 +396,7 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
     c0 = __reduce_add_sync(0xffffffffu, c0);
     if (CW == 2) c1 = __reduce_add_sync(0xffffffffu, c1);
     if (lane == 0) { s_cnt[par][0][warp] = c0; if (CW == 2) s_cnt[par][1][warp] = c1; }
-    team_sync();
+    if (real) team_sync();
     const uint4 v = *reinterpret_cast<const uint4 *>(&s_cnt[par][0][0]);
     n0 = v.x + v.y + v.z + v.w;
     n1 = 0;
@@ -388,7 +406,6 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
     }
     par ^= 1;
   };
-  uint32_t theta = 0u;
   {
     const uint32_t t = 1u << 30;
     uint32_t c = 0, n0, n1;
@@ -411,7 +428,9 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
     const uint32_t na = n0 & ((1u << SH) - 1), nb = (n0 >> SH) & ((1u << SH) - 1), nc = (CW == 1) ? (n0 >> SH2) : n1;
     if (na >= ku) theta = ta; else if (nb >= ku) theta = tb; else if (nc >= ku) theta = tc;
   }
+  }
   COBS_SEL_STAMP(4);
+  if (real || part == 3) {
   // keep every key above theta and the lowest-index `need_eq` keys equal to it, in index order: one scan of the
   // packed (above, equal) counts gives both the totals and this thread's position
   int v = 0;
@@ -425,7 +444,7 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
     if (lane >= o) inc += t;
   }
   if (lane == 31) s_scan[warp] = inc;
-  team_sync();
+  if (real) team_sync();
   int base = 0, total = 0;
 #pragma unroll
   for (int q = 0; q < kSelWarps; ++q) { const int t = s_scan[q]; total += t; base += (q < warp) ? t : 0; }
@@ -439,8 +458,9 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
       bool keep = false;
       if (keys[j] > theta) keep = true;
       else if (keys[j] == theta) { keep = eq_rank < need_eq; ++eq_rank; }
-      if (keep && pos >= 0 && pos < k) out[pos++] = b0 + j;
+      if (keep && pos >= 0 && pos < k && !dry) out[pos++] = b0 + j;
     }
+  }
   }
   COBS_SEL_STAMP(5);
 }
@@ -451,33 +471,46 @@ template <int PPC>
 __device__ void select_team(const Params &p, const int *seq_lens, int tid, int count_mult, int empty_need) {
   __shared__ int s_ok;
   const int units = p.B * p.Hkv;
-  for (int u = blockIdx.x; u < units; u += gridDim.x) {
+  // The first pass over the first unit is a rehearsal: the same code on whatever the workspace holds, nothing written,
+  // run while the unit is still being scored, each of the team's four warps taking one quarter of it.  The
+  // selection is executed once or twice per CTA and launch, so its instructions are never in the SM's instruction
+  // cache when it is needed, and after other work has swept L2 they come from HBM, one dependent miss after
+  // another (measured: 16 us for a selection that takes 5 us once its code is near); rehearsed in four parallel
+  // pieces, the real pass finds them close by.
+  bool rehearsal = true;
+  for (int u = blockIdx.x; u < units;) {
     const int T = seq_lens[u / p.Hkv];
     const int n_sum = min(T / p.L, p.NB);
     const int n_cand = min(window_start(T, p.window, p.L) / p.L, n_sum);
     const int n_chunks = (n_sum + 15) / 16;
-    if (tid == 0) {
-      int ok = 0;
-      for (long long it = 0; it < kSpinLimit; ++it) {
-        if (ld_volatile(p.ctl_score + u) >= (n_chunks > 0 ? n_chunks * count_mult : empty_need)) { ok = 1; break; }
-        __nanosleep(200);
+    if (!rehearsal) {
+      if (tid == 0) {
+        int ok = 0;
+        for (long long it = 0; it < kSpinLimit; ++it) {
+          if (ld_volatile(p.ctl_score + u) >= (n_chunks > 0 ? n_chunks * count_mult : empty_need)) { ok = 1; break; }
+          __nanosleep(200);
+        }
+        if (!ok) report(p.status, COBS_ERR_TIMEOUT);
+        s_ok = ok;
       }
-      if (!ok) report(p.status, COBS_ERR_TIMEOUT);
-      s_ok = ok;
+      team_sync();
+      const int ok = s_ok;
+      team_sync();
+      if (!ok) { u += gridDim.x; continue; }     // never scored: leave the unit unselected (its attention times out too)
+      __threadfence();
+      COBS_SEL_STAMP(0);
     }
+    const int part = rehearsal ? (tid >> 5) : -1;
+    if (n_sum <= kSelThreads * 4) select_unit<PPC, 4>(p, u, n_sum, n_cand, tid, part);
+    else if (n_sum <= kSelThreads * 8) select_unit<PPC, 8>(p, u, n_sum, n_cand, tid, part);
+    else select_unit<PPC, 16>(p, u, n_sum, n_cand, tid, part);
     team_sync();
-    const int ok = s_ok;
-    team_sync();
-    if (!ok) continue;                         // never scored: leave the unit unselected (its attention times out too)
-    __threadfence();
-    COBS_SEL_STAMP(0);
-    if (n_sum <= kSelThreads * 4) select_unit<PPC, 4>(p, u, n_sum, n_cand, tid);
-    else if (n_sum <= kSelThreads * 8) select_unit<PPC, 8>(p, u, n_sum, n_cand, tid);
-    else select_unit<PPC, 16>(p, u, n_sum, n_cand, tid);
+    if (rehearsal) { rehearsal = false; continue; }
     __threadfence();
     team_sync();
     if (tid == 0) atomicExch(p.ctl_ready + u, 1);
     COBS_SEL_STAMP(1);
+    u += gridDim.x;
   }
 }
 
