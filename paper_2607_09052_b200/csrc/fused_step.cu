@@ -350,11 +350,11 @@ __device__ void select_unit(const Params &p, int u, int n_sum, int n_cand, int t
           for (int q = 0; q < kSelWarps; ++q) M = fmaxf(M, s_m[g][q]);
           float S = 0.f;
 #pragma unroll
-          for (int q = 0; q < kSelWarps; ++q) S += (s_m[g][q] == -INFINITY) ? 0.f : s_s[g][q] * expf(s_m[g][q] - M);
-          const float lse = M + logf(S);
+          for (int q = 0; q < kSelWarps; ++q) S += (s_m[g][q] == -INFINITY) ? 0.f : s_s[g][q] * __expf(s_m[g][q] - M);
+          const float lse = M + __logf(S);              // fast forms: a few instructions instead of dozens (this code runs cold)
 #pragma unroll
           for (int q = 0; q < NQ; ++q) {
-            const float wq = (own_m[g][q] != -INFINITY) ? expf(own_m[g][q] - lse) : 0.f;
+            const float wq = (own_m[g][q] != -INFINITY) ? __expf(own_m[g][q] - lse) : 0.f;
             sc[4 * q + 0] = fmaf(x[gg][q].x, wq, sc[4 * q + 0]); sc[4 * q + 1] = fmaf(x[gg][q].y, wq, sc[4 * q + 1]);
             sc[4 * q + 2] = fmaf(x[gg][q].z, wq, sc[4 * q + 2]); sc[4 * q + 3] = fmaf(x[gg][q].w, wq, sc[4 * q + 3]);
           }
