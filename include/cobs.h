@@ -53,7 +53,7 @@ typedef enum {
   COBS_ERR_UNSUPPORTED = 2,         /* a shape this build has no kernel for */
   COBS_ERR_WORKSPACE_TOO_SMALL = 3,
   COBS_ERR_CUDA = 4,                /* a CUDA runtime call failed (launch configuration, copy) */
-  COBS_ERR_TIMEOUT = 5,             /* device status: a bounded device-side wait ran out */
+  COBS_ERR_TIMEOUT = 5,             /* device status: a bounded device-side wait ran out; the call's outputs are undefined */
   COBS_ERR_BOUNDS = 6               /* device status: a page id or block index was out of range and skipped */
 } cobs_status;
 

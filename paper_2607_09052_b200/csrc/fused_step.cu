@@ -569,8 +569,10 @@ __device__ __forceinline__ void fp4_rows_full_width(uint32_t xa, uint32_t xb, ui
 // DT: COBS_SUMM_BF16 | COBS_SUMM_FP4_E2M1.  WPT: 32-bit words of codes per thread per FP4 row
 // (Ds_pad / 32).  NT: f16 terms of the query (1: full space, 2: fp32 subspace query).
 // ---------------------------------------------------------------------------------------------------
+// Returns false when a wait for this warp's own copies ran out (COBS_ERR_TIMEOUT is recorded): copies may then still
+// be on their way into the warp's ring, so the caller must not reuse it.
 template <int DT, int D, int WPT, int NT>
-__device__ void score_phase(const Params &p, const int *seq_lens, unsigned char *wsm, uint64_t *bars, int wg, int n_wg,
+__device__ bool score_phase(const Params &p, const int *seq_lens, unsigned char *wsm, uint64_t *bars, int wg, int n_wg,
                             int lane) {
   constexpr bool FP4 = (DT == COBS_SUMM_FP4_E2M1);
   constexpr int MCH = D / 32;                 // 16-byte chunks of a bf16 row per thread
@@ -981,6 +983,7 @@ __device__ void score_phase(const Params &p, const int *seq_lens, unsigned char 
   }
   COBS_ACC(0);
   COBS_ACC_FLUSH(1200 + wg);
+  return alive;
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1804,10 +1807,12 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
     }
     __syncwarp();
     COBS_STAMP(0);
-    if (phases & PH_SCORE) score_phase<DT, D, WPT, NT>(p, seq_lens, wsm, &s_bars[warp][0], wg, n_wg, lane);
+    bool ring_free = true;
+    if (phases & PH_SCORE) ring_free = score_phase<DT, D, WPT, NT>(p, seq_lens, wsm, &s_bars[warp][0], wg, n_wg, lane);
     COBS_STAMP(1);
     COBS_STAMP(2);
-    if (phases & PH_ATTEND) attend_phase<D>(p, seq_lens, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
+    // after a timeout in scoring the step's outputs are undefined; this warp leaves its items to the others
+    if ((phases & PH_ATTEND) && ring_free) attend_phase<D>(p, seq_lens, wsm, wg, n_wg, lane, (phases & PH_SCORE) != 0);
     COBS_STAMP(3);
   } else if (phases & PH_SCORE) {
     // ---- selection team ----------------------------------------------------------------------------------------
