@@ -5,17 +5,16 @@
 //   C      = K~ K~^T / L      (L x L Gram matrix)             (Method, Cost: Gram trick)
 //   (lambda_i, w_i) = eigenpairs of C, lambda descending
 //   xi_i   = K~^T w_i / sqrt(L)  = sqrt(lambda_i) u_i         (Eq. lowrank)
-// computed without forming C: one-sided (Hestenes) Jacobi rotates pairs of ROWS of K~ until all rows are mutually
-// orthogonal.  The product of the rotations is W^T, so the rows end up as K~^T w_i = sqrt(L) xi_i with squared
-// norms L lambda_i: the same O(L^2 D) work per sweep as the Gram route, the L x L matrices never exist, and a
-// rotation is one dot product and one update of two rows held by a warp.
+// Only the r largest eigenpairs are wanted: C is tridiagonalised by Householder reflections, the r largest
+// eigenvalues are located by Sturm counts, their eigenvectors come from inverse iteration and are carried back
+// through the reflections (the builder's comment below has the details).  A block whose eigenvectors fail their
+// residual check is solved by one-sided (Hestenes) Jacobi instead: pairs of ROWS of K~ are rotated until all rows
+// are mutually orthogonal; the product of the rotations is W^T, so the rows end up as K~^T w_i = sqrt(L) xi_i with
+// squared norms L lambda_i.
 //   store  : fp32 | bf16 (RNE) | FP4 E2M1 + one scale per factor (Method, Quantization)
 //
 // One CTA per (sequence, KV head, block); everything stays in shared memory.  All reductions run in
 // a fixed order, so the output bits are a function of the input bits only.
-#ifdef COBS_BUILD_DEBUG
-#include <cstdio>
-#endif
 #include "common.cuh"
 
 namespace cobs {
@@ -307,15 +306,17 @@ __global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel
   // Kc <- the block's keys as fp32, minus their mean; first: the mean (fixed summation order) is computed and stored,
   // and the mean squared norm; project: K~ <- K~ U_Q (one warp per row, in place).
   auto load_keys = [&](bool first, bool project) {
-    for (int c = tid; c < L * (D / 2); c += kBuildThreads) {
-      const int t = c / (D / 2), dp = c - t * (D / 2);
+#pragma unroll 4
+    for (int c = tid; c < L * (D / 8); c += kBuildThreads) {        // 16 bytes (8 keys' elements) per thread and turn
+      const int t = c / (D / 8), d8 = c - t * (D / 8);
       const int tok = blk * L + t;
-      int pg = p.page_table[(size_t)b_idx * p.mpp + tok / p.P];
-      uint32_t w = 0;
+      const int pg = p.page_table[(size_t)b_idx * p.mpp + tok / p.P];
+      uint4 w = make_uint4(0u, 0u, 0u, 0u);
       if (pg < 0 || pg >= p.n_pages) report(p.status, COBS_ERR_BOUNDS);
-      else w = reinterpret_cast<const uint32_t *>(p.k_pages)[((((size_t)pg * p.Hkv + h) * p.P + (tok % p.P)) * D) / 2 + dp];
-      Kc[t * ldk + 2 * dp] = bf16_lo(w);
-      Kc[t * ldk + 2 * dp + 1] = bf16_hi(w);
+      else w = reinterpret_cast<const uint4 *>(p.k_pages + (((size_t)pg * p.Hkv + h) * p.P + (tok % p.P)) * D)[d8];
+      float *dst = Kc + t * ldk + 8 * d8;
+      *reinterpret_cast<float4 *>(dst) = make_float4(bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y));
+      *reinterpret_cast<float4 *>(dst + 4) = make_float4(bf16_lo(w.z), bf16_hi(w.z), bf16_lo(w.w), bf16_hi(w.w));
     }
     __syncthreads();
     if (first) {
@@ -380,16 +381,9 @@ __global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel
   const int r_eff = min(p.r, L);
   int *s_fallback = reinterpret_cast<int *>(lam + 40);
   bool use_jacobi = solver == 1;
-#ifdef COBS_BUILD_DEBUG
-  const long long t0 = clock64();
-  long long t2 = t0, t3 = t0, t4 = t0, t5 = t0;
-#endif
   if (!use_jacobi) {
     if (tid == 0) *s_fallback = 0;
     gram_tridiag<TL>(Kc, ldk, Dk4, Ct, dd, ee, bet, xrow, dgl, pp, lam + 48, tid, warp, lane);
-#ifdef COBS_BUILD_DEBUG
-    t2 = clock64();
-#endif
 
     // ---- the r largest eigenvalues of T: Gershgorin bounds, then every warp narrows one eigenvalue 32 ways per step ----
     if (warp == 0) {
@@ -445,9 +439,6 @@ __global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel
       }
     }
     __syncthreads();
-#ifdef COBS_BUILD_DEBUG
-    t3 = clock64();
-#endif
 
     // ---- eigenvectors of T by inverse iteration ---------------------------------------------------------------------
     // (T - s I) = P L U with row interchanges, by lane 0 of the vector's warp: the reciprocal of U's diagonal, its two
@@ -478,13 +469,13 @@ __global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel
                 float p0 = swp ? sub : a0;
                 const float p1 = swp ? nd : a1, p2 = swp ? ne : 0.f;
                 if (fabsf(p0) < pivmin) p0 = copysignf(pivmin, p0);
-                const float inv = 1.0f / p0, mlt = (swp ? a0 : sub) * inv;
+                const float inv = __fdividef(1.0f, p0), mlt = (swp ? a0 : sub) * inv;   // (a rounding error here only moves the shift)
                 u1[i] = p1; u2[i] = p2; iv[i] = inv; mm[i] = mlt; sw[i] = swp ? 1.f : 0.f;
                 a0 = (swp ? a1 : nd) - mlt * p1;
                 a1 = (swp ? 0.f : ne) - mlt * p2;
               }
               if (fabsf(a0) < pivmin) a0 = copysignf(pivmin, a0);
-              iv[L - 1] = 1.0f / a0; u1[L - 1] = 0.f; u2[L - 1] = 0.f;
+              iv[L - 1] = __fdividef(1.0f, a0); u1[L - 1] = 0.f; u2[L - 1] = 0.f;
             }
             __syncwarp();
           }
@@ -555,9 +546,6 @@ __global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel
         __syncthreads();
       }
     }
-#ifdef COBS_BUILD_DEBUG
-    t4 = clock64();
-#endif
     // ---- check |T z - lambda z| (and that z is a unit vector); a failure sends the block to the Jacobi solver ----------
     for (int j = warp; j < r_eff; j += NW) {
       if (top[j] < 0) continue;
@@ -573,9 +561,6 @@ __global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel
     }
     __syncthreads();
     use_jacobi = *s_fallback != 0;
-#ifdef COBS_BUILD_DEBUG
-    t5 = clock64();
-#endif
     if (!use_jacobi) {
       back_transform<TL>(Z, Ct, bet, top, r_eff, warp, lane);      // w = Q z
       __syncthreads();
@@ -733,10 +718,6 @@ __global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel
   __syncthreads();
   }
 
-#ifdef COBS_BUILD_DEBUG
-  const long long t6 = clock64();
-  if (tid == 0 && (use_jacobi || blockIdx.x % 4096 == 7)) printf("DBG blk %d jac %d gram+tri %lld eig %lld inv %lld chk %lld back+xi %lld\n", (int)blockIdx.x, (int)use_jacobi, t2-t0, t3-t2, t4-t3, t5-t4, t6-t5);
-#endif
   // ---- sign rule + store, one warp per factor ---------------------------------------------------------
   for (int i = warp; i < p.r; i += NW) {
     float *row = xi_s + i * Dk;

@@ -837,6 +837,87 @@ def test_builder_cfg5_like_block128():
     check_builder(WL["cfg5_64k_g8"].replace(batch=1, seq_len=4096), [(0, 4)])
 
 
+@pytest.mark.parametrize("case", ["cfg1_tiny", "cfg4_like", "cfg5_like", "subspace"])
+def test_builder_jacobi_route(case, monkeypatch):
+    """The builder's second eigen-solver (taken by a block whose tridiagonal route fails its residual check), forced
+    for every block: the same checks against the oracle's definitions."""
+    monkeypatch.setenv("COBS_BUILD_SOLVER", "jacobi")
+    if case == "cfg1_tiny":
+        check_builder(WL["cfg1_tiny"], [(0, 0)])
+    elif case == "cfg4_like":
+        check_builder(WL["cfg4_128k"].replace(batch=1, seq_len=2048), [(0, 3)])
+    elif case == "cfg5_like":
+        check_builder(WL["cfg5_64k_g8"].replace(batch=1, seq_len=2048), [(0, 4)])
+    else:
+        check_builder(WL["cfg3a_32k_subspace"].replace(batch=1, seq_len=1024), [(0, 2)])
+
+
+@pytest.mark.parametrize("solver", ["tridiagonal", "jacobi"])
+@pytest.mark.parametrize("L", [16, 32, 64, 128])
+def test_builder_structured_spectra(L, solver, monkeypatch):
+    """Blocks whose Gram matrices are not generic: rank one, two equal leading eigenvalues, a few distinct tokens
+    repeated (a reducible tridiagonal form), a spectrum of well separated and of nearly equal eigenvalues, tokens
+    equal in pairs.  Errors are measured against the largest eigenvalue (backward error): factors of numerically
+    null directions are rounding noise in fp32 and exact zeros in the oracle's fp64."""
+    if solver == "jacobi":
+        monkeypatch.setenv("COBS_BUILD_SOLVER", "jacobi")
+    B = _binding()
+    D, r, nblk = 64, 4, 6
+    wl = WL["cfg1_tiny"].replace(block_size=L, page_size=16, seq_len=nblk * L, window=L, topk=2, rank=r)
+    cpu = synth.generate(wl)
+    g = torch.Generator().manual_seed(1234 + L)
+    blocks = []
+    u = torch.linalg.qr(torch.randn(D, D, generator=g))[0]                       # orthonormal directions
+    t = torch.randn(L, generator=g)
+    blocks.append(1.5 + t[:, None] * u[:, 0][None, :] * 2.0)                     # rank one
+    a = torch.linalg.qr(torch.randn(L, 2, generator=g) - 0.0)[0]
+    a = a - a.mean(0, keepdim=True)
+    a = torch.linalg.qr(a)[0] * (L ** 0.5)
+    blocks.append(a[:, :1] * u[:, 1][None, :] + a[:, 1:2] * u[:, 2][None, :] + 0.01 * torch.randn(L, D, generator=g))  # two equal
+    few = torch.randn(3, D, generator=g)
+    blocks.append(few[torch.arange(L) % 3])                                      # three distinct tokens
+    sv = torch.tensor([4.0, 2.0, 1.0, 0.5] + [0.01] * (D - 4))
+    blocks.append(torch.randn(L, D, generator=g) @ (u * sv[None, :]).T)          # separated
+    sv = torch.tensor([1.0, 0.9999, 0.9998, 0.5, 0.4999] + [0.05] * (D - 5))
+    blocks.append(torch.randn(L, D, generator=g) @ (u * sv[None, :]).T)          # nearly equal
+    half = torch.randn(L // 2, D, generator=g)
+    blocks.append(half.repeat_interleave(2, dim=0))                              # tokens equal in pairs
+    kp = cpu["k_pages"]                                                          # [n_pages][Hkv][P][D]
+    assert kp.shape[1] == 1 and kp.shape[3] == D
+    ppb = L // wl.page_size
+    for i, blk in enumerate(blocks):
+        pages = cpu["page_table"][0, i * ppb:(i + 1) * ppb].long()
+        kp[pages, 0] = blk.to(torch.bfloat16).reshape(ppb, wl.page_size, D)
+    inp = to_dev(cpu)
+    cfg = B.make_config(wl)
+    s = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    B.cobs_build_summaries(cfg, B.make_kv(inp), 0, wl.max_blocks, s, ws)
+    assert B.cobs_read_status(ws) == 0
+    _, xi, _ = B.summary_views(cfg, s)
+    K, _ = synth.unit_kv(cpu, wl, 0, 0)
+    K = K.numpy()
+    for i in range(nblk):
+        kb = K[i * L:(i + 1) * L]
+        _, sigma = O.block_mean_and_covariance(kb)
+        lam = np.sort(np.linalg.eigvalsh(sigma))[::-1]
+        lam0 = lam[0]
+        x = xi[0, 0, i].double().cpu().numpy()
+        for f in range(r):
+            n2 = x[f] @ x[f]
+            assert abs(n2 - lam[f]) <= 2e-5 * lam0, (i, f, n2, lam[f])
+            assert np.linalg.norm(sigma @ x[f] - n2 * x[f]) <= 1e-4 * lam0 * np.sqrt(lam0), (i, f)
+            for f2 in range(f):
+                assert abs(x[f] @ x[f2]) <= 1e-4 * lam0, (i, f, f2)
+        # the rank-r approximation the scorer uses, as a matrix
+        approx = x.T @ x
+        w, v = np.linalg.eigh(sigma)
+        want = (v[:, -r:] * w[-r:]) @ v[:, -r:].T
+        gap = lam[r - 1] - lam[r]
+        slack = 2e-4 * lam0 + (gap if gap < 1e-3 * lam0 else 0.0)
+        assert np.linalg.norm(approx - want, 2) <= slack, (i, np.linalg.norm(approx - want, 2), slack)
+
+
 def test_builder_constant_key_block_gives_zero_factors():
     B = _binding()
     wl = WL["cfg1_tiny"].replace(summary_dtype="fp4")
