@@ -853,6 +853,17 @@ def test_builder_jacobi_route(case, monkeypatch):
 
 
 @pytest.mark.parametrize("solver", ["tridiagonal", "jacobi"])
+@pytest.mark.parametrize("rank,L,D", [(12, 64, 128), (16, 128, 64), (15, 32, 64)])
+def test_builder_ranks_above_eight(rank, L, D, solver, monkeypatch):
+    """More factors than the builder has warps: two eigenvectors per warp in the inverse iteration."""
+    if solver == "jacobi":
+        monkeypatch.setenv("COBS_BUILD_SOLVER", "jacobi")
+    wl = synth.Workload("highrank", 1, 4, 2, D, 6 * L, L, 16, rank=rank, topk=2, window=L, summary_dtype="fp32",
+                        key_model="block_offset", planted=1, shuffle_pages=True, seed=21)
+    check_builder(wl, [(0, 0), (0, 1)])
+
+
+@pytest.mark.parametrize("solver", ["tridiagonal", "jacobi"])
 @pytest.mark.parametrize("L", [16, 32, 64, 128])
 def test_builder_structured_spectra(L, solver, monkeypatch):
     """Blocks whose Gram matrices are not generic: rank one, two equal leading eigenvalues, a few distinct tokens
