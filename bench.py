@@ -314,7 +314,8 @@ def run_phase_times(args):
     out["scoring_working_warps"] = int(busy.sum())
     if not score_only:
         at = raw[:, :n].astype(np.float64) / mhz
-        names_a = ["draw item", "item set-up", "wait for selection", "group table + query", "stream loop", "write partial", "close + merge"]
+        names_a = ["after the draw", "item set-up", "wait for selection", "group table + query", "stream loop",
+                   "write partial + fence + count", "draw the next item", "merge (last closer of a unit)"]
         out["attention_us_per_warp"] = {nm: round(float(at[k].mean()), 2) for k, nm in enumerate(names_a)}
         late = np.argsort(t[3])[-8:]
         out["latest_warps"] = [{"warp": int(w), "attention_start": round(float((t[2][w] - t0) / 1e3), 1),

@@ -1035,6 +1035,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     int last = 0;
     if (lane == 0) last = (atomicAdd(p.ctl_att + u, 1) + 1 == n_splits);
     last = __shfl_sync(0xffffffffu, last, 0);
+    COBS_ACC(5);
     if (!last) return;
     // ---- merge the unit's partials: o = sum_s e^{m_s - M} acc_s / sum_s e^{m_s - M} l_s -------------------
     // A slice is [G][D] accumulators followed by [G] (max, sum) pairs.  Few round trips: all pairs at once, then the
@@ -1295,7 +1296,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
                make_float2((l_run > 0.f) ? m_run * (sl2 * 0.6931471805599453f) : -INFINITY, l_run));
     }
     close_item(u);
-    COBS_ACC(5);
+    COBS_ACC(7);
     int next_item = 0;
     if (lane == 0) next_item = atomicAdd(p.ctl_item, 1);
     item = __shfl_sync(0xffffffffu, next_item, 0);
