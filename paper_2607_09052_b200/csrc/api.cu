@@ -110,7 +110,7 @@ static WorkspaceLayout layout_workspace(const cobs_config *c) {
   const size_t B = c->batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, G = Hq / Hkv, D = c->head_dim;
   size_t off = 0;
   w.status = off; off += kStatusBytes;
-  w.ctl = off; off = align_up(off + 3 * B * Hkv * sizeof(int), 256);     // inside the first kCtlBytes
+  w.ctl = off; off = align_up(off + 6 * B * Hkv * sizeof(int), 256);     // two sets of three counters per unit, inside the first kCtlBytes
   w.e = off; off = align_up(off + B * Hq * (size_t)c->max_blocks * sizeof(float), 256);
   w.lse_part = off; off = align_up(off + B * Hq * (size_t)((c->max_blocks + 15) / 16) * 4 * 2 * sizeof(float), 256);   // up to four pairs per chunk
   w.partial = off; off = align_up(off + B * Hkv * (size_t)choose_splits(c) * G * (D + 2) * sizeof(float), 256);
@@ -136,7 +136,7 @@ static void fill_params(Params &p, const cobs_config *c, void *workspace) {
     WorkspaceLayout w = layout_workspace(c);
     char *base = static_cast<char *>(workspace);
     p.status = reinterpret_cast<int32_t *>(base + w.status);
-    p.ctl_done = reinterpret_cast<int *>(base + w.status) + 1;
+    p.ctl_epoch = reinterpret_cast<int *>(base + w.status) + 1;
     p.ctl_item = reinterpret_cast<int *>(base + w.status) + 2;
     p.ctl_bar = reinterpret_cast<int *>(base + w.status) + 3;
     p.ctl_score = reinterpret_cast<int *>(base + w.ctl);

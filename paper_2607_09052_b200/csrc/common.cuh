@@ -13,7 +13,7 @@ namespace cobs {
 constexpr int kStatusBytes = 256;          // status word lives in the first 256 bytes of the workspace
 constexpr int kMaxSplits = 64;             // upper bound on split-KV partials per (sequence, KV head)
 constexpr int kMaxUnits = 65535;           // (sequence, KV head) units a workspace has counters for
-constexpr int kCtlBytes = kStatusBytes + 3 * kMaxUnits * 4;   // status word + counters, zeroed by cobs_reset_status
+constexpr int kCtlBytes = kStatusBytes + 6 * kMaxUnits * 4;   // status block + two sets of counters, zeroed by cobs_reset_status
 
 // Everything a kernel needs, passed by value.
 struct Params {
@@ -33,7 +33,9 @@ struct Params {
   float *skew;                // optional [B][Hkv][NB][r] fp32: third-cumulant scalar per stored factor (full-space descriptors)
   // workspace pieces
   int32_t *status;
-  int *ctl_done;              // CTAs of the persistent kernel that have finished
+  // hand-off counters of the persistent kernel: two sets, used by alternate launches (bit 31 of the epoch word names
+  // the set of the next launch; set 1 lies 3 ints after set 0 for the two words, 3 * B * Hkv ints for the arrays)
+  int *ctl_epoch;             // set of the next launch (bit 31) | CTAs of the running launch that have begun
   int *ctl_item;              // next attention item to hand out
   int *ctl_bar;               // CTAs that have passed the grid barrier after the query projection
   int *ctl_score;             // [B * Hkv] scored chunks per unit

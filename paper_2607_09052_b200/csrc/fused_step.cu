@@ -57,6 +57,31 @@ constexpr int kFThreads = (kFWarps + kSelWarps) * 32;        // one CTA per SM
 constexpr int kScoreStageBytes = 14080;                      // means + factor rows + scales of a 16-block chunk
 constexpr int kAttStages = 3;
 constexpr int kAttStageBytes = 2 * 16 * 128 * 2;             // K + V of one 16-token group, D = 128
+// The hand-off counters exist twice.  A launch works on the set named by bit 31 of the epoch word; the low bits of
+// that word count the CTAs that have begun.  The CTA that begins last (every other CTA then holds its set number) turns
+// the word over for the next launch and clears the other set, which the previous launch left dirty: nothing has to
+// be cleaned up when the kernel ends, and a launch that gave up half-way does not poison the next one.
+__shared__ int s_ctl[3];          // offset of this launch's per-unit counters, of its item / barrier words; "begun last"
+#define CTL_UNIT(ptr) ((ptr) + s_ctl[0])
+#define CTL_MISC(ptr) ((ptr) + s_ctl[1])
+__device__ __forceinline__ void ctl_begin(const Params &p) {          // thread 0 of every CTA, before the CTA's first barrier
+  const unsigned old = atomicAdd(reinterpret_cast<unsigned *>(p.ctl_epoch), 1u);
+  const int set = (int)(old >> 31);
+  s_ctl[0] = set * 3 * p.B * p.Hkv;
+  s_ctl[1] = set * 3;
+  s_ctl[2] = (old & 0x7fffffffu) == gridDim.x - 1;
+}
+__device__ __forceinline__ void ctl_turn(const Params &p) {           // the whole CTA that began last, after that barrier
+  const int units = p.B * p.Hkv;
+  const int other_u = s_ctl[0] ? 0 : 3 * units, other_m = s_ctl[1] ? 0 : 3;
+  if (threadIdx.x == 0) {
+    atomicAdd(reinterpret_cast<unsigned *>(p.ctl_epoch), 0x80000000u - gridDim.x);     // flips bit 31, zeroes the count
+    p.ctl_item[other_m] = 0;
+    p.ctl_bar[other_m] = 0;
+  }
+  for (int i = threadIdx.x; i < 3 * units; i += blockDim.x) p.ctl_score[other_u + i] = 0;   // score, ready, att: contiguous
+}
+
 constexpr int kTableEntries = 256;                           // 16-token groups per attention item
 constexpr int kRingBytes = (2 * kScoreStageBytes > kAttStages * kAttStageBytes + kTableEntries * 8)
                                ? 2 * kScoreStageBytes : kAttStages * kAttStageBytes + kTableEntries * 8;
@@ -487,7 +512,7 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid, int c
       if (tid == 0) {
         int ok = 0;
         for (long long it = 0; it < kSpinLimit; ++it) {
-          if (ld_volatile(p.ctl_score + u) >= (n_chunks > 0 ? n_chunks * count_mult : empty_need)) { ok = 1; break; }
+          if (ld_volatile(CTL_UNIT(p.ctl_score) + u) >= (n_chunks > 0 ? n_chunks * count_mult : empty_need)) { ok = 1; break; }
           __nanosleep(200);
         }
         if (!ok) report(p.status, COBS_ERR_TIMEOUT);
@@ -508,7 +533,7 @@ __device__ void select_team(const Params &p, const int *seq_lens, int tid, int c
     if (rehearsal) { rehearsal = false; continue; }
     __threadfence();
     team_sync();
-    if (tid == 0) atomicExch(p.ctl_ready + u, 1);
+    if (tid == 0) atomicExch(CTL_UNIT(p.ctl_ready) + u, 1);
     COBS_SEL_STAMP(1);
     u += gridDim.x;
   }
@@ -605,7 +630,7 @@ __device__ bool score_phase(const Params &p, const int *seq_lens, unsigned char 
   const uint32_t ring = (uint32_t)__cvta_generic_to_shared(wsm);
   const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
   const float inv_sqrt_d = 1.0f / sqrtf((float)D);
-  const float ln_l = logf((float)L);
+  const float ln_l = (float)(31 - __clz(L)) * 0.6931471805599453f;      // L is a power of two
 
   // Work order.  The units are scored in kWaves waves (first half, second half); within a wave every streaming
   // warp takes one contiguous range of the wave's chunks (mostly one unit: its query fragments are built once, and
@@ -782,10 +807,11 @@ __device__ bool score_phase(const Params &p, const int *seq_lens, unsigned char 
             }
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            int ex = 0;
-            if (mx > 0.f) frexpf(mx, &ex);
-            const float inv_s = ldexpf(1.0f, 1 - ex);       // power of two bringing max |q| into [1, 2)
-            const float mult = ldexpf(1.0f, ex - 1) * (p.qtilde ? 1.0f : inv_sqrt_d);
+            // mx in [2^(ex-1), 2^ex), from its exponent field (clamped: an all-zero or absurdly large query keeps
+            // the powers of two below in range)
+            const int ex = (int)(__float_as_uint(fminf(fmaxf(mx, 1e-30f), 1e30f)) >> 23) - 126;
+            const float inv_s = __uint_as_float((uint32_t)(128 - ex) << 23);       // 2^(1-ex): brings max |q| into [1, 2)
+            const float mult = __uint_as_float((uint32_t)(126 + ex) << 23) * (p.qtilde ? 1.0f : inv_sqrt_d);
 #pragma unroll
             for (int j = 0; j < WPT; ++j) {
 #pragma unroll
@@ -929,7 +955,7 @@ __device__ bool score_phase(const Params &p, const int *seq_lens, unsigned char 
       if (pend_u != u && pend_n > 0) {       // moving on to another unit: count the finished one's chunks
         __threadfence();
         __syncwarp();
-        if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
+        if (lane == 0) atomicAdd(CTL_UNIT(p.ctl_score) + pend_u, pend_n);
         pend_n = 0;
         COBS_ACC(7);
       }
@@ -979,7 +1005,7 @@ __device__ bool score_phase(const Params &p, const int *seq_lens, unsigned char 
   if (pend_n > 0) {
     __threadfence();
     __syncwarp();
-    if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
+    if (lane == 0) atomicAdd(CTL_UNIT(p.ctl_score) + pend_u, pend_n);
   }
   COBS_ACC(0);
   COBS_ACC_FLUSH(1200 + wg);
@@ -1001,7 +1027,8 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
   constexpr int NCP = (16 * CH) / 32;         // cp.async per lane per operand per stage
   const int gid = lane >> 2, tig = lane & 3;
   const int G = p.G, L = p.L, P = p.P, units = p.B * p.Hkv, n_splits = p.n_splits;
-  const int gpb = L / 16;
+  const int lgL = 31 - __clz(L), lgP = 31 - __clz(P), lgg = lgL - 4;      // L and P are powers of two: shifts, not divisions
+  const int gpb = L >> 4;
   const uint32_t ring = (uint32_t)__cvta_generic_to_shared(wsm);
   uint32_t *goff = reinterpret_cast<uint32_t *>(wsm + kAttStages * kAttStageBytes);
   int *gtok = reinterpret_cast<int *>(goff + kTableEntries);
@@ -1033,7 +1060,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     __threadfence();
     __syncwarp();
     int last = 0;
-    if (lane == 0) last = (atomicAdd(p.ctl_att + u, 1) + 1 == n_splits);
+    if (lane == 0) last = (atomicAdd(CTL_UNIT(p.ctl_att) + u, 1) + 1 == n_splits);
     last = __shfl_sync(0xffffffffu, last, 0);
     COBS_ACC(5);
     if (!last) return;
@@ -1046,7 +1073,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     const float *pu = p.partial + (size_t)u * n_splits * SL;
     float *sm_w = reinterpret_cast<float *>(wsm);            // [n_splits][G] maxima, then weights
     float *sm_l = sm_w + kMaxSplits * 8;        // [n_splits][G] sums
-    float *sm_M = sm_l + kMaxSplits * 8;        // [8] maxima, [8] denominators
+    float *sm_M = sm_l + kMaxSplits * 8;        // [8] maxima, [8] denominators, [8] their reciprocals
     for (int base = 0; base < np; base += 128) {
       float2 pv[4];
 #pragma unroll
@@ -1076,7 +1103,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
       }
       dn += __shfl_xor_sync(0xffffffffu, dn, 8);
       dn += __shfl_xor_sync(0xffffffffu, dn, 16);
-      if (sub == 0 && g < G) { sm_M[g] = mx; sm_M[8 + g] = dn; }
+      if (sub == 0 && g < G) { sm_M[g] = mx; sm_M[8 + g] = dn; sm_M[16 + g] = 1.0f / dn; }
     }
     __syncwarp();
     constexpr int KV = 4 * D / 64;                           // float2 per lane for four heads
@@ -1111,21 +1138,21 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
         const int idx = lane + 32 * k;
         if (idx < nv2) {
           const int head = gq + idx / (D / 2), col = (idx - (idx / (D / 2)) * (D / 2)) * 2;
-          const float den = sm_M[8 + head];
+          const float inv = sm_M[16 + head];            // one division per head; the rows are scaled by its result
           const size_t bh = (size_t)b_idx * p.Hq + h * G + head;
-          *reinterpret_cast<float2 *>(p.out + bh * D + col) = make_float2(acc[k].x / den, acc[k].y / den);
+          *reinterpret_cast<float2 *>(p.out + bh * D + col) = make_float2(acc[k].x * inv, acc[k].y * inv);
         }
       }
       if (p.lse && lane < min(4, G - gq)) {
         const int head = gq + lane;
-        p.lse[(size_t)b_idx * p.Hq + h * G + head] = sm_M[head] + logf(sm_M[8 + head]);
+        p.lse[(size_t)b_idx * p.Hq + h * G + head] = sm_M[head] + __logf(sm_M[8 + head]);
       }
     }
     __syncwarp();
   };
 
   int item = 0;
-  if (lane == 0) item = atomicAdd(p.ctl_item, 1);
+  if (lane == 0) item = atomicAdd(CTL_MISC(p.ctl_item), 1);
   item = __shfl_sync(0xffffffffu, item, 0);
   for (;;) {
     COBS_ACC(0);
@@ -1134,8 +1161,8 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     const int b_idx = u / p.Hkv, h = u - b_idx * p.Hkv;
     const int T = seq_lens[b_idx];
     const int ws = window_start(T, p.window, L);
-    const int n_cand = ws / L;
-    const int n_win = (T - ws + L - 1) / L;
+    const int n_cand = ws >> lgL;
+    const int n_win = (T - ws + L - 1) >> lgL;
     int n_sel = min(p.topk, n_cand);
     const int n_groups_u = (n_sel + n_win) * gpb;
     const int per = (n_groups_u + n_splits - 1) / n_splits;
@@ -1156,7 +1183,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     COBS_ACC(1);
     if (g0 < n_sel * gpb && n_groups > 0) {
       if (wait_select) {
-        ok = wait_flag(p.ctl_ready + u);
+        ok = wait_flag(CTL_UNIT(p.ctl_ready) + u);
         if (!ok && lane == 0) report(p.status, COBS_ERR_TIMEOUT);
         __threadfence();
       } else {
@@ -1167,7 +1194,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     // ---- table of this item's groups -----------------------------------------------------------------
     __syncwarp();
     for (int g = lane; g < n_groups; g += 32) {
-      const int gg = g0 + g, it = gg / gpb, sub = gg - it * gpb;
+      const int gg = g0 + g, it = gg >> lgg, sub = gg - (it << lgg);
       int blk;
       bool good = ok;
       if (it < min(p.topk, n_cand)) {          // a selected-block slot
@@ -1181,10 +1208,10 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
       int first = -1;
       uint32_t off = 0;
       if (good && tok0 < T) {
-        const int pslot = tok0 / P;                                  // a length beyond the page-table row is not followed
+        const int pslot = tok0 >> lgP;                                // a length beyond the page-table row is not followed
         const int pg = (pslot < p.mpp) ? p.page_table[(size_t)b_idx * p.mpp + pslot] : -1;
         if (pg < 0 || pg >= p.n_pages) report(p.status, COBS_ERR_BOUNDS);
-        else { first = tok0; off = (uint32_t)(((((size_t)pg * p.Hkv + h) * P + (tok0 % P)) * D) / 8); }
+        else { first = tok0; off = (uint32_t)(((((size_t)pg * p.Hkv + h) * P + (tok0 & (P - 1))) * D) / 8); }
       }
       goff[g] = off;
       gtok[g] = first;
@@ -1298,7 +1325,7 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     close_item(u);
     COBS_ACC(7);
     int next_item = 0;
-    if (lane == 0) next_item = atomicAdd(p.ctl_item, 1);
+    if (lane == 0) next_item = atomicAdd(CTL_MISC(p.ctl_item), 1);
     item = __shfl_sync(0xffffffffu, next_item, 0);
     COBS_ACC(6);
   }
@@ -1587,7 +1614,7 @@ __device__ void umma_epilogue(const Params &p, const UmmaList &l, unsigned char 
     if (pend_n > 0) {
       __threadfence();
       __syncwarp();
-      if (lane == 0) atomicAdd(p.ctl_score + pend_u, pend_n);
+      if (lane == 0) atomicAdd(CTL_UNIT(p.ctl_score) + pend_u, pend_n);
       pend_n = 0;
     }
   };
@@ -1765,10 +1792,10 @@ __device__ void grid_barrier(const Params &p) {
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
-    atomicAdd(p.ctl_bar, 1);
+    atomicAdd(CTL_MISC(p.ctl_bar), 1);
     bool ok = false;
     for (long long it = 0; it < kSpinLimit; ++it) {
-      if (ld_volatile(p.ctl_bar) >= (int)gridDim.x) { ok = true; break; }
+      if (ld_volatile(CTL_MISC(p.ctl_bar)) >= (int)gridDim.x) { ok = true; break; }
       __nanosleep(50);
     }
     if (!ok) report(p.status, COBS_ERR_TIMEOUT);
@@ -1789,11 +1816,13 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
   // sequence lengths are consulted at every change of unit: keep them in shared memory when they fit
   __shared__ int s_len[kLenCache];
   const int *seq_lens = p.seq_lens;
+  if (threadIdx.x == 0) ctl_begin(p);          // (its round trip overlaps the loads of the lengths)
   if (p.B <= kLenCache) {
     for (int i = threadIdx.x; i < p.B; i += kFThreads) s_len[i] = p.seq_lens[i];
     seq_lens = s_len;
   }
   __syncthreads();
+  if (s_ctl[2]) ctl_turn(p);
   if ((phases & PH_SCORE) && p.u_q) {
     project_queries(p);
     grid_barrier(p);
@@ -1819,19 +1848,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_step_kernel(Params p, int 
     // ---- selection team ----------------------------------------------------------------------------------------
     select_team<1>(p, seq_lens, (int)threadIdx.x - kFWarps * 32, 1, 1);
   }
-  // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
-  __syncthreads();
-  __shared__ int is_last;
-  if (threadIdx.x == 0) {
-    __threadfence();
-    is_last = (atomicAdd(p.ctl_done, 1) + 1 == (int)gridDim.x);
-  }
-  __syncthreads();
-  if (is_last) {
-    const int units = p.B * p.Hkv;
-    for (int i = threadIdx.x; i < units; i += kFThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
-    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; *p.ctl_bar = 0; }
-  }
+  // (nothing to clean up: the next launch works on the other set of counters, see ctl_begin)
 }
 
 // The step with phase S on tcgen05 (packed E2M1, full key space, D = 128, r = 8); phases must include PH_SCORE.
@@ -1856,6 +1873,7 @@ __global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p,
     for (int i = 0; i < kUAccBufs; ++i) { mbar_init(bars + (kBTFull + i) * 8, 1); mbar_init(bars + (kBTEmpty + i) * 8, 4); }
     mbar_init(bars + kBTiles * 8, kSelWarps);
     s_abort = 0;
+    ctl_begin(p);
     umma_list_make(s_list, p.B * p.Hkv, p.NB, (int)gridDim.x, (int)blockIdx.x);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -1867,6 +1885,7 @@ __global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p,
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (s_ctl[2]) ctl_turn(p);
   const uint32_t tmem = s_tmem;
   volatile int *abort_flag = &s_abort;
   if (warp < kFWarps) {
@@ -1886,23 +1905,12 @@ __global__ void __launch_bounds__(kUThreads, 1) fused_step_umma_kernel(Params p,
   } else {
     umma_issuer(p, s_list, fsm, bars, tmem, lane, abort_flag);
   }
-  // ---- the last CTA to finish puts the counters back to zero for the next call --------------------------
+  // ---- the tensor memory goes back when every role is done (the counters need no clean-up, see ctl_begin) -------
   tc_fence_before();
   __syncthreads();
-  __shared__ int is_last;
-  if (threadIdx.x == 0) {
-    __threadfence();
-    is_last = (atomicAdd(p.ctl_done, 1) + 1 == (int)gridDim.x);
-  }
   if (warp == kFWarps + kSelWarps + 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kUAccCols * kUAccBufs));
-  }
-  __syncthreads();
-  if (is_last) {
-    const int units = p.B * p.Hkv;
-    for (int i = threadIdx.x; i < units; i += kUThreads) { p.ctl_score[i] = 0; p.ctl_ready[i] = 0; p.ctl_att[i] = 0; }
-    if (threadIdx.x == 0) { *p.ctl_done = 0; *p.ctl_item = 0; *p.ctl_bar = 0; }
   }
 }
 
@@ -2079,16 +2087,16 @@ extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void 
   Params p;
   int32_t st = prepare_attend_params(cfg, q, kv, sel_idx, sel_cnt, out, lse_or_null, &p);
   if (st != COBS_OK) return st;
-  // scratch layout: [status word + launch counter: 256 B][3 counters per unit][split partials]
+  // scratch layout: [status word, epoch word, item / barrier words: 256 B][two sets of 3 counters per unit][split partials]
   const size_t units = (size_t)p.B * p.Hkv;
-  const size_t ctl_bytes = (3 * units * sizeof(int) + 255) / 256 * 256;
+  const size_t ctl_bytes = (6 * units * sizeof(int) + 255) / 256 * 256;
   const size_t partial_bytes = units * p.n_splits * p.G * (size_t)(p.D + 2) * sizeof(float);
   if (kStatusBytes + ctl_bytes + partial_bytes > (size_t)COBS_STATIC_SCRATCH_BYTES) return COBS_ERR_WORKSPACE_TOO_SMALL;
   cudaError_t e = cudaSuccess;
   unsigned char *base = static_cast<unsigned char *>(static_scratch_address(&e));
   if (!base) return COBS_ERR_CUDA;
   p.status = reinterpret_cast<int32_t *>(base);
-  p.ctl_done = reinterpret_cast<int *>(base) + 1;
+  p.ctl_epoch = reinterpret_cast<int *>(base) + 1;
   p.ctl_item = reinterpret_cast<int *>(base) + 2;
   p.ctl_bar = reinterpret_cast<int *>(base) + 3;
   p.ctl_score = reinterpret_cast<int *>(base + kStatusBytes);
