@@ -735,6 +735,45 @@ def test_length_beyond_the_page_table_is_reported_not_followed():
     assert B.cobs_read_status(ws) == 0
 
 
+def test_step_replays_from_a_cuda_graph():
+    """The fused step captured once and replayed: its hand-off counters alternate between two sets by themselves
+    (no host state), so odd and even replays give the bits of a plain call; the status word stays clear."""
+    B = _binding()
+    wl = WL["cfg2_32k"].replace(seq_len=8192)
+    inp = to_dev(synth.generate(wl))
+    cfg = B.make_config(wl)
+    kv = B.make_kv(inp)
+    summ = B.SummaryBuffers(cfg, "cuda")
+    ws = B.alloc_workspace(cfg, "cuda")
+    B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, summ, ws)
+    nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+    out = torch.zeros((nb, hq, D), dtype=torch.float32, device="cuda")
+    lse = torch.zeros((nb, hq), dtype=torch.float32, device="cuda")
+    sel = torch.zeros((nb, hkv, wl.topk), dtype=torch.int32, device="cuda")
+    cnt = torch.zeros((nb, hkv), dtype=torch.int32, device="cuda")
+    B.cobs_decode_step(cfg, inp["q"], kv, summ, out, lse, sel, cnt, ws)
+    torch.cuda.synchronize()
+    ref_out, ref_sel, ref_lse = out.clone(), sel.clone(), lse.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        B.cobs_decode_step(cfg, inp["q"], kv, summ, out, lse, sel, cnt, ws)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            B.cobs_decode_step(cfg, inp["q"], kv, summ, out, lse, sel, cnt, ws)
+    for _ in range(5):
+        out.zero_(); sel.zero_(); lse.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref_out) and torch.equal(sel, ref_sel) and torch.equal(lse, ref_lse)
+    # and a plain call after the replays
+    out.zero_()
+    B.cobs_decode_step(cfg, inp["q"], kv, summ, out, lse, sel, cnt, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref_out)
+    assert B.cobs_read_status(ws) == 0
+
+
 # --- builder (backward error; eigenvectors of close eigenvalues are not unique to rounding) ---------------------
 
 def check_builder(wl, units):
