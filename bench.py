@@ -37,7 +37,7 @@ from paper_2607_09052_b200 import shard, synth  # noqa: E402
 DEFAULT_WORKLOAD = "cfg4_128k"
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused kernel (ncu; see profiles/)
-TRAFFIC_BYTES = {"cfg4_128k": 4 * (128266240 + 3536896)}   # batch-4 capture x 4 (traffic is proportional to batch)
+TRAFFIC_BYTES = {"cfg4_128k": 4 * (128485376 + 3605760)}   # batch-4 capture x 4 (traffic is proportional to batch)
 
 
 def algorithmic_bytes(wl: synth.Workload, record_bytes: int) -> int:
