@@ -16,7 +16,10 @@
  *   - Every pointer is a DEVICE pointer owned by the caller unless a parameter is named *_host.
  *     The library allocates no device memory and frees none; scratch comes from the caller as
  *     `workspace` (size from cobs_workspace_bytes, 256-byte aligned).  The workspace must not be
- *     shared by calls that may overlap on the GPU.
+ *     shared by calls that may overlap on the GPU.  Calls of different configurations may use one
+ *     workspace in turn if it is as large as the largest of them needs (the first 1.5 MB hold the
+ *     status word and the hand-off counters of the persistent kernel, at the same places for every
+ *     shape; cobs_reset_status clears them).
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
  *     the call returns without synchronising, except the *_host entry point and cobs_read_status.
  *   - Arguments are validated on the host before anything is launched; a call that returns a

@@ -110,7 +110,10 @@ static WorkspaceLayout layout_workspace(const cobs_config *c) {
   const size_t B = c->batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, G = Hq / Hkv, D = c->head_dim;
   size_t off = 0;
   w.status = off; off += kStatusBytes;
-  w.ctl = off; off = align_up(off + 6 * B * Hkv * sizeof(int), 256);     // two sets of three counters per unit, inside the first kCtlBytes
+  // two sets of three counters per unit.  The area has the size of the largest shape (1.5 MB) and set 1 starts
+  // 3 * kMaxUnits ints after set 0 whatever the shape, so that a workspace that serves calls of different shapes keeps
+  // its counters in the same places and no call's scratch arrays lie over another shape's counters
+  w.ctl = off; off = align_up(off + 6 * (size_t)kMaxUnits * sizeof(int), 256);
   w.e = off; off = align_up(off + B * Hq * (size_t)c->max_blocks * sizeof(float), 256);
   w.lse_part = off; off = align_up(off + B * Hq * (size_t)((c->max_blocks + 15) / 16) * 4 * 2 * sizeof(float), 256);   // up to four pairs per chunk
   w.partial = off; off = align_up(off + B * Hkv * (size_t)choose_splits(c) * G * (D + 2) * sizeof(float), 256);
@@ -140,6 +143,7 @@ static void fill_params(Params &p, const cobs_config *c, void *workspace) {
     p.ctl_item = reinterpret_cast<int *>(base + w.status) + 2;
     p.ctl_bar = reinterpret_cast<int *>(base + w.status) + 3;
     p.ctl_score = reinterpret_cast<int *>(base + w.ctl);
+    p.ctl_set_stride = 3 * kMaxUnits;
     p.ctl_ready = p.ctl_score + (size_t)p.B * p.Hkv;
     p.ctl_att = p.ctl_ready + (size_t)p.B * p.Hkv;
     p.qtilde_out = reinterpret_cast<float *>(base + w.qtilde);

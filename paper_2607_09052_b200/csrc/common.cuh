@@ -34,13 +34,14 @@ struct Params {
   // workspace pieces
   int32_t *status;
   // hand-off counters of the persistent kernel: two sets, used by alternate launches (bit 31 of the epoch word names
-  // the set of the next launch; set 1 lies 3 ints after set 0 for the two words, 3 * B * Hkv ints for the arrays)
+  // the set of the next launch; set 1 lies 3 ints after set 0 for the two words, ctl_set_stride ints for the arrays)
   int *ctl_epoch;             // set of the next launch (bit 31) | CTAs of the running launch that have begun
   int *ctl_item;              // next attention item to hand out
   int *ctl_bar;               // CTAs that have passed the grid barrier after the query projection
   int *ctl_score;             // [B * Hkv] scored chunks per unit
   int *ctl_ready;             // [B * Hkv] 1 once the unit's selection is written
   int *ctl_att;               // [B * Hkv] attention slices finished per unit
+  int ctl_set_stride;         // ints from a per-unit array of set 0 to the same array of set 1 (the same for every shape)
   const float *qtilde;        // [B][Hq][Ds_pad] projected subspace query (what the scoring reads), or NULL
   float *qtilde_out;          // where the step kernel's prologue writes it (workspace)
   float *e;                   // [B][Hkv][G][NB]

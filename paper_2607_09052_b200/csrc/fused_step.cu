@@ -59,27 +59,33 @@ constexpr int kAttStages = 3;
 constexpr int kAttStageBytes = 2 * 16 * 128 * 2;             // K + V of one 16-token group, D = 128
 // The hand-off counters exist twice.  A launch works on the set named by bit 31 of the epoch word; the low bits of
 // that word count the CTAs that have begun.  The CTA that begins last (every other CTA then holds its set number) turns
-// the word over for the next launch and clears the other set, which the previous launch left dirty: nothing has to
-// be cleaned up when the kernel ends, and a launch that gave up half-way does not poison the next one.
-__shared__ int s_ctl[3];          // offset of this launch's per-unit counters, of its item / barrier words; "begun last"
+// the word over for the next launch and clears the other set, which the previous launch left dirty (as far as that
+// launch's unit count reached: the word after the epoch word keeps it, so a workspace may serve calls of different
+// shapes).  Nothing has to be cleaned up when the kernel ends, and a launch that gave up half-way does not poison
+// the next one.  Status block, in ints: 0 status, 1 epoch, 2 / 3 item and barrier words of set 0, 4 extent, 5 / 6
+// item and barrier words of set 1.
+__shared__ int s_ctl[4];          // offset of this launch's per-unit counters, of its item / barrier words; "begun last"; extent
 #define CTL_UNIT(ptr) ((ptr) + s_ctl[0])
 #define CTL_MISC(ptr) ((ptr) + s_ctl[1])
 __device__ __forceinline__ void ctl_begin(const Params &p) {          // thread 0 of every CTA, before the CTA's first barrier
   const unsigned old = atomicAdd(reinterpret_cast<unsigned *>(p.ctl_epoch), 1u);
   const int set = (int)(old >> 31);
-  s_ctl[0] = set * 3 * p.B * p.Hkv;
+  s_ctl[0] = set * p.ctl_set_stride;
   s_ctl[1] = set * 3;
   s_ctl[2] = (old & 0x7fffffffu) == gridDim.x - 1;
 }
 __device__ __forceinline__ void ctl_turn(const Params &p) {           // the whole CTA that began last, after that barrier
-  const int units = p.B * p.Hkv;
-  const int other_u = s_ctl[0] ? 0 : 3 * units, other_m = s_ctl[1] ? 0 : 3;
+  const int other_u = s_ctl[0] ? 0 : p.ctl_set_stride, other_m = s_ctl[1] ? 0 : 3;
   if (threadIdx.x == 0) {
+    s_ctl[3] = min(*reinterpret_cast<const volatile int *>(p.ctl_epoch + 3), p.ctl_set_stride);   // ints of the other set its last launch used
     atomicAdd(reinterpret_cast<unsigned *>(p.ctl_epoch), 0x80000000u - gridDim.x);     // flips bit 31, zeroes the count
     p.ctl_item[other_m] = 0;
     p.ctl_bar[other_m] = 0;
   }
-  for (int i = threadIdx.x; i < 3 * units; i += blockDim.x) p.ctl_score[other_u + i] = 0;   // score, ready, att: contiguous
+  __syncthreads();
+  const int ext = s_ctl[3];
+  for (int i = threadIdx.x; i < ext; i += blockDim.x) p.ctl_score[other_u + i] = 0;     // score, ready, att: contiguous
+  if (threadIdx.x == 0) p.ctl_epoch[3] = 3 * p.B * p.Hkv;             // what this launch will leave behind in its set
 }
 
 constexpr int kTableEntries = 256;                           // 16-token groups per attention item
@@ -2087,9 +2093,9 @@ extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void 
   Params p;
   int32_t st = prepare_attend_params(cfg, q, kv, sel_idx, sel_cnt, out, lse_or_null, &p);
   if (st != COBS_OK) return st;
-  // scratch layout: [status word, epoch word, item / barrier words: 256 B][two sets of 3 counters per unit][split partials]
+  // scratch layout: [status word, epoch word, item / barrier words: 256 B][3 counters per unit][split partials]
   const size_t units = (size_t)p.B * p.Hkv;
-  const size_t ctl_bytes = (6 * units * sizeof(int) + 255) / 256 * 256;
+  const size_t ctl_bytes = (3 * units * sizeof(int) + 255) / 256 * 256;     // every call starts from cleared words: set 0 only
   const size_t partial_bytes = units * p.n_splits * p.G * (size_t)(p.D + 2) * sizeof(float);
   if (kStatusBytes + ctl_bytes + partial_bytes > (size_t)COBS_STATIC_SCRATCH_BYTES) return COBS_ERR_WORKSPACE_TOO_SMALL;
   cudaError_t e = cudaSuccess;
@@ -2099,6 +2105,7 @@ extern "C" int32_t cobs_sparse_decode_static(const cobs_config *cfg, const void 
   p.ctl_epoch = reinterpret_cast<int *>(base) + 1;
   p.ctl_item = reinterpret_cast<int *>(base) + 2;
   p.ctl_bar = reinterpret_cast<int *>(base) + 3;
+  p.ctl_set_stride = 0;                       // (the extent word is cleared with the rest: the other set is never touched)
   p.ctl_score = reinterpret_cast<int *>(base + kStatusBytes);
   p.ctl_ready = p.ctl_score + units;
   p.ctl_att = p.ctl_ready + units;

@@ -735,6 +735,46 @@ def test_length_beyond_the_page_table_is_reported_not_followed():
     assert B.cobs_read_status(ws) == 0
 
 
+def test_one_workspace_serves_calls_of_different_shapes():
+    """A workspace as large as the largest of three shapes needs, used by their steps in a mixed order: every step
+    gives the bits it gives on a workspace of its own (the hand-off counters of the persistent kernel live at the same
+    places for every shape, and each launch clears what the previous one left, however many units that one had)."""
+    B = _binding()
+
+    def setup(wl):
+        inp = to_dev(synth.generate(wl))
+        cfg = B.make_config(wl)
+        kv = B.make_kv(inp)
+        summ = B.SummaryBuffers(cfg, "cuda")
+        own = B.alloc_workspace(cfg, "cuda")
+        B.cobs_build_summaries(cfg, kv, 0, wl.max_blocks, summ, own)
+        nb, hq, hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+        x = dict(wl=wl, inp=inp, cfg=cfg, kv=kv, summ=summ,
+                 out=torch.zeros((nb, hq, D), dtype=torch.float32, device="cuda"),
+                 lse=torch.zeros((nb, hq), dtype=torch.float32, device="cuda"),
+                 sel=torch.zeros((nb, hkv, wl.topk), dtype=torch.int32, device="cuda"),
+                 cnt=torch.zeros((nb, hkv), dtype=torch.int32, device="cuda"))
+        B.cobs_decode_step(cfg, inp["q"], kv, summ, x["out"], x["lse"], x["sel"], x["cnt"], own)
+        torch.cuda.synchronize()
+        x["ref_out"], x["ref_sel"] = x["out"].clone(), x["sel"].clone()
+        return x
+
+    a = setup(WL["cfg2_32k"].replace(seq_len=8192, batch=4))                      # 32 units
+    b = setup(WL["cfg2_32k"].replace(seq_len=4096, batch=1))                      # 8 units
+    c = setup(WL["cfg4_128k"].replace(seq_len=4096, batch=9))                     # 72 units, another descriptor
+    size = max(B.cobs_workspace_bytes(x["cfg"]) for x in (a, b, c))
+    raw = torch.zeros(size + 256, dtype=torch.uint8, device="cuda")
+    off = (-raw.data_ptr()) % 256
+    ws = raw[off:off + size]
+    B.cobs_reset_status(ws)
+    for x in (a, b, c, a, a, c, b, b, a, c, b, a):
+        x["out"].zero_(); x["sel"].zero_()
+        B.cobs_decode_step(x["cfg"], x["inp"]["q"], x["kv"], x["summ"], x["out"], x["lse"], x["sel"], x["cnt"], ws)
+        torch.cuda.synchronize()
+        assert torch.equal(x["out"], x["ref_out"]) and torch.equal(x["sel"], x["ref_sel"])
+        assert B.cobs_read_status(ws) == 0
+
+
 def test_step_replays_from_a_cuda_graph():
     """The fused step captured once and replayed: its hand-off counters alternate between two sets by themselves
     (no host state), so odd and even replays give the bits of a plain call; the status word stays clear."""
