@@ -278,7 +278,7 @@ __host__ __device__ inline BuildSmem build_smem_layout(const Params &p) {
 }
 
 template <int TL>
-__global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 3) build_kernel(Params p, int block_begin, int block_end, int solver) {
+__global__ void __launch_bounds__(kBuildThreads, (TL == 8) ? 2 : 4) build_kernel(Params p, int block_begin, int block_end, int solver) {
   extern __shared__ __align__(16) float sm[];
   constexpr int L = 16 * TL;
   const int D = p.D, Dk = p.Ds, ldk = build_ldk(p);
