@@ -79,10 +79,10 @@ __global__ void quantise_kernel(const float *xi, long long n_vectors, int Ds, in
 // --- Gram matrix and Householder tridiagonalisation in registers -----------------------------------------------
 // The 256 threads form a 16 x 16 grid; thread (ty, tx) keeps the elements (ty + 16 a, tx + 16 b) of the symmetric
 // matrix, a, b < TL = L / 16, in registers (a cyclic layout: the trailing matrix of every step is spread evenly, and
-// whole groups a or b that lie in the finished part are skipped).  Step k: every warp forms the reflector v of row k
-// from a copy of that row in shared memory, the threads multiply their tiles by v and reduce over the 16 threads of
+// whole groups a or b that lie in the finished part are skipped).  Step k: the 16 threads that own row k have left
+// its reflector v in shared memory, the threads multiply their tiles by v and reduce over the 16 threads of
 // a matrix row (p = beta A v), then apply A <- A - v w^T - w v^T with w = p - (beta v^T p / 2) v.  The threads that
-// own row k + 1 publish their rows for the next step.  Two barriers per step.
+// own row k + 1 publish their rows and form the next reflector.  Two barriers per step.
 // Out: dd / ee (diagonal and off-diagonal of T), bet (2 / v^T v, 0 where a row needed no reflector), and the
 // reflectors packed row after row in Ct (row k: its L - 1 - k elements right of the diagonal).
 __host__ __device__ constexpr int refl_offset(int k, int L) { return k * (L - 1) - k * (k - 1) / 2; }
@@ -112,37 +112,49 @@ __device__ __forceinline__ void gram_tridiag(const float *__restrict__ Kc, int l
     }
   }
   __syncthreads();                                    // the keys have been read: their place is free for the reflectors
-  // a published row k has zeros up to its diagonal (column k included): it is the reflector but for the element k + 1
-  if (ty == 0) {
+  // The 16 threads that own row `row` publish their TL rows (zeros up to the diagonal, column `row` included), then
+  // turn the published row into its reflector v: sigma = |x|^2 over the 16 lanes, alpha = -sign(x0) sqrt(sigma),
+  // beta = 1 / (sigma - x0 alpha), v = x with x0 - alpha as its first element.  bet[row] = 0: the row needs no reflector.
+  auto publish = [&](int row, float *xn) {
+    if (ty != (row & 15)) return;
+    const unsigned mask = 0xffffu << (16 * (ty & 1));          // the half-warp of these threads
 #pragma unroll
     for (int a = 0; a < TL; ++a)
 #pragma unroll
-      for (int b = 0; b < TL; ++b) xrow[a * L + tx + 16 * b] = (tx + 16 * b > 0) ? A[a][b] : 0.f;
-  }
+      for (int b = 0; b < TL; ++b) xn[a * L + tx + 16 * b] = (tx + 16 * b > row) ? A[a][b] : 0.f;
+    if (row + 2 >= L) return;                                  // the last two rows are only read, not reduced
+    __syncwarp(mask);
+    float *xr = xn + (row >> 4) * L;
+    float sg = 0.f;
+#pragma unroll
+    for (int b = 0; b < TL; ++b) { const float x = xr[tx + 16 * b]; sg = fmaf(x, x, sg); }
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) sg += __shfl_xor_sync(mask, sg, o);
+    const float x0 = xr[row + 1];
+    const bool refl = sg - x0 * x0 > 1e-30f + 1e-14f * sg;
+    const float alpha = refl ? -copysignf(sqrtf(sg), x0) : x0;
+    const float beta = refl ? 1.0f / (sg - x0 * alpha) : 0.f;
+    __syncwarp(mask);                                          // everyone has read x0
+    if (tx == 0) {
+      ee[row] = alpha; bet[row] = beta;
+      if (refl) xr[row + 1] = x0 - alpha;
+    }
+  };
+  publish(0, xrow);
   if (ty == tx) {
 #pragma unroll
     for (int a = 0; a < TL; ++a) dgl[ty + 16 * a] = A[a][a];
   }
   __syncthreads();
   for (int k = 0; k + 2 < L; ++k) {
-    const float *xc = xrow + (k & 1) * TL * L + (k >> 4) * L;
+    const float *xc = xrow + (k & 1) * TL * L + (k >> 4) * L;      // the reflector of row k
     float *xn = xrow + ((k + 1) & 1) * TL * L;
     const int amin = (k + 1) >> 4;                    // groups below hold finished rows / columns only
-    float sg = 0.f;
-    for (int c = lane; c < L; c += 32) { const float x = xc[c]; sg = fmaf(x, x, sg); }
-    sg = warp_sum(sg);
-    const float x0 = xc[k + 1];
-    const bool refl = sg - x0 * x0 > 1e-30f + 1e-14f * sg;         // (uniform: every warp computes the same numbers)
-    const float alpha = refl ? -copysignf(sqrtf(sg), x0) : x0;
-    const float beta = refl ? 1.0f / (sg - x0 * alpha) : 0.f;
-    if (tid == 0) { ee[k] = alpha; bet[k] = beta; }
-    if (refl) {
+    const float beta = bet[k];
+    if (beta != 0.f) {                                // (uniform)
       float vr[TL], vc[TL];
 #pragma unroll
-      for (int a = 0; a < TL; ++a) {
-        vr[a] = xc[ty + 16 * a] - ((ty + 16 * a == k + 1) ? alpha : 0.f);
-        vc[a] = xc[tx + 16 * a] - ((tx + 16 * a == k + 1) ? alpha : 0.f);
-      }
+      for (int a = 0; a < TL; ++a) { vr[a] = xc[ty + 16 * a]; vc[a] = xc[tx + 16 * a]; }
       if (ty == 0) {
 #pragma unroll
         for (int b = 0; b < TL; ++b)
@@ -191,12 +203,7 @@ __device__ __forceinline__ void gram_tridiag(const float *__restrict__ Kc, int l
       for (int b = 0; b < TL; ++b)
         if (tx + 16 * b > k) Ct[refl_offset(k, L) + tx + 16 * b - k - 1] = 0.f;
     }
-    if (ty == ((k + 1) & 15)) {                     // all TL rows of these threads; the readers take row (k + 1) / 16
-#pragma unroll
-      for (int a = 0; a < TL; ++a)
-#pragma unroll
-        for (int b = 0; b < TL; ++b) xn[a * L + tx + 16 * b] = (tx + 16 * b > k + 1) ? A[a][b] : 0.f;
-    }
+    publish(k + 1, xn);
     if (ty == tx) {
 #pragma unroll
       for (int a = 0; a < TL; ++a) dgl[ty + 16 * a] = A[a][a];
