@@ -35,8 +35,9 @@
 //
 // Cross-warp hand-offs go through global counters in the workspace (release: write, __threadfence,
 // atomicAdd; acquire: volatile read, __threadfence, .cg loads).  Every wait is bounded; on expiry the
-// kernel records COBS_ERR_TIMEOUT, skips the dependent work and returns.  The last CTA to finish puts
-// the counters back to zero, so a workspace needs zeroing only once (cobs_reset_status).
+// kernel records COBS_ERR_TIMEOUT, skips the dependent work and returns.  The counters come in two sets
+// that alternate launches take turns on (ctl_begin), so a workspace needs zeroing only once
+// (cobs_reset_status) and nothing is cleaned up when the kernel ends.
 #include <cuda.h>
 #include <cuda_fp8.h>
 
