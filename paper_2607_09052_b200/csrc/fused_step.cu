@@ -1172,8 +1172,9 @@ __device__ void attend_phase(const Params &p, const int *seq_lens, unsigned char
     const int n_win = (T - ws + L - 1) >> lgL;
     int n_sel = min(p.topk, n_cand);
     const int n_groups_u = (n_sel + n_win) * gpb;
-    const int per = (n_groups_u + n_splits - 1) / n_splits;
-    const int g0 = min(split * per, n_groups_u), g1 = min(g0 + per, n_groups_u);
+    // slices of equal size to within one group (ceil-sized slices would leave the last slice of a unit nearly empty
+    // and make every other one longer)
+    const int g0 = (split * n_groups_u) / n_splits, g1 = ((split + 1) * n_groups_u) / n_splits;
     int n_groups = min(g1 - g0, kTableEntries);
     // ---- query fragments: rows = heads (zero padded to 16), natural k order.
     // Loaded first: the loads fly while the warp waits for the unit's selection and builds its group table.
